@@ -1,0 +1,176 @@
+/*
+ * decentlam.h -- C ABI of the B200 (sm_100a) DecentLaM update library.
+ *
+ * One GPU simulates all n nodes of a decentralised data-parallel job.  The parameter
+ * replicas x, the momenta m and the stochastic gradients g of the n nodes are stacked
+ * row-wise as [n, d] arrays in device memory (row i = node i, Sec. 4 / App. A notation
+ * "x = [x_1; ...; x_n]").  One call performs one iteration k -> k+1 for every node at once.
+ *
+ * General rules for every entry point
+ *   - Returns DLM_OK (0) or a negative dlm_status; nothing is printed, thrown or aborted.
+ *   - Pointers marked "device" must be device memory of the current CUDA device; pointers
+ *     marked "host" are ordinary host memory.  The caller owns every buffer it passes.
+ *   - The step functions and lsq_grad only enqueue work on `cuda_stream` (a cudaStream_t
+ *     cast to void*, NULL = default stream) and return; results are valid once the stream
+ *     reaches that point.  They never synchronise, never allocate and never wait on device
+ *     memory inside a kernel.
+ *   - All arguments are validated on the host before anything is launched.
+ */
+#ifndef DECENTLAM_H_
+#define DECENTLAM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dlm_status {
+    DLM_OK = 0,
+    DLM_ERR_NULL = -1,        /* a required pointer is NULL */
+    DLM_ERR_SHAPE = -2,       /* n < 1, d < 1, ld < d, p/q < 1, n mismatch with the topology ... */
+    DLM_ERR_ALIGN = -3,       /* a pointer is not aligned to its element size */
+    DLM_ERR_ALIAS = -4,       /* x, m and g (or A, b, x, g) overlap */
+    DLM_ERR_HYPER = -5,       /* gamma not finite or <= 0; beta outside [0, 1) */
+    DLM_ERR_KIND = -6,        /* unknown topology kind or gradient dtype */
+    DLM_ERR_TOPOLOGY = -7,    /* CSR input violates the documented requirements */
+    DLM_ERR_UNSUPPORTED = -8, /* n above DLM_MAX_NODES, or a size the kernels cannot tile */
+    DLM_ERR_CUDA = -9,        /* a CUDA runtime/driver call failed (launch, copy, alloc) */
+    DLM_ERR_WORKSPACE = -10   /* workspace missing, misaligned or too small */
+} dlm_status;
+
+/* Human-readable name of a status code; never NULL. */
+const char* dlm_status_string(int status);
+
+/* ------------------------------------------------------------------------------------
+ * Topology: the weight matrix W = [w_ij] of Sec. 3 ("Network topology and weights"),
+ * w_ij > 0 iff j is in the neighbourhood N_i (which contains i).  Stored per time slot
+ * as CSR: rowptr int32[n+1], col int32[nnz] ascending within a row, val fp32[nnz].
+ * Row i lists the nodes j that node i receives from, with weight w_ij.
+ *
+ * Weight rule for the built-in kinds: every off-diagonal weight is 1/q for an integer q,
+ * computed in double and rounded once to fp32; the diagonal is the fp32 rounding of
+ * 1 - sum_{j != i} 1/q_ij (double, ascending j).
+ * ------------------------------------------------------------------------------------ */
+typedef struct dlm_topology dlm_topology;
+
+typedef enum dlm_topology_kind {
+    DLM_TOPO_RING = 0,         /* N_i = {i-1, i, i+1} mod n, weights 1/3 (App. G "Ring"); n >= 3 */
+    DLM_TOPO_STATIC_EXP = 1,   /* i receives from (i + 2^t) mod n, t = 0..L-1, L = floor(log2(n-1))+1;
+                                  all L+1 weights 1/(L+1); directed; n >= 2 */
+    DLM_TOPO_ONE_PEER_EXP = 2, /* period L; in slot t node i receives from (i + 2^t) mod n only,
+                                  weights 1/2 and 1/2; n >= 2 */
+    DLM_TOPO_COMPLETE = 3,     /* w_ij = 1/n (Sec. 3: the fully connected case) */
+    DLM_TOPO_CSR_MH = 4,       /* caller gives an undirected graph, weights by the Metropolis-Hastings
+                                  rule cited under Assumption A.3: w_ij = 1/(1 + max(deg_i, deg_j)) */
+    DLM_TOPO_CSR_WEIGHTS = 5   /* caller gives W itself */
+} dlm_topology_kind;
+
+#define DLM_MAX_NODES 2048
+
+/*
+ * Build the tables for a topology on n nodes and upload them to the current device.
+ *   rowptr, col, val : host; used only by the CSR kinds, ignored (may be NULL) otherwise.
+ *     DLM_TOPO_CSR_MH      rowptr[n+1], col[]: adjacency lists WITHOUT self loops, ascending,
+ *                          no duplicates, symmetric (j in list i <=> i in list j); val ignored.
+ *     DLM_TOPO_CSR_WEIGHTS rowptr[n+1], col[], val[]: ascending, no duplicates, self entry
+ *                          present in every row, weights > 0, every row sum and every column
+ *                          sum within 1e-6 of 1 (doubly stochastic, Assumption A.3).
+ *   out : receives the handle.  The library owns it (host and device tables) until
+ *         topology_destroy.  The inputs are copied; the caller may free them at once.
+ * Errors: DLM_ERR_NULL, DLM_ERR_KIND, DLM_ERR_SHAPE (n too small for the kind),
+ *         DLM_ERR_UNSUPPORTED (n > DLM_MAX_NODES), DLM_ERR_TOPOLOGY, DLM_ERR_CUDA.
+ */
+int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
+                   dlm_topology** out);
+
+/* Number of distinct slots; iteration k uses slot k mod period (k = 0 is the first step). */
+int topology_period(const dlm_topology* topo, int* period);
+
+/* Number of nodes the topology was built for. */
+int topology_nodes(const dlm_topology* topo, int* n);
+
+/* Borrowed pointers to the CSR tables of one slot, valid until topology_destroy.
+ * _host returns host pointers, _device device pointers.  Any out-pointer may be NULL.
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE (slot outside [0, period)). */
+int topology_tables_host(const dlm_topology* topo, int slot, const int32_t** rowptr,
+                         const int32_t** col, const float** val, int64_t* nnz);
+int topology_tables_device(const dlm_topology* topo, int slot, const int32_t** rowptr,
+                           const int32_t** col, const float** val, int64_t* nnz);
+
+/* Free host and device tables.  NULL is accepted. */
+int topology_destroy(dlm_topology* topo);
+
+/* ------------------------------------------------------------------------------------
+ * Update rules.  Common arguments:
+ *   topo      : weights; slot k mod period is used.
+ *   k         : iteration counter (>= 0), only selects the slot.
+ *   n, d      : nodes (must equal the topology's n) and coordinates per node.
+ *   x, m      : device fp32 [n, d], row stride ld elements (ld >= d); updated IN PLACE.
+ *   g         : device [n, d], row stride ldg elements; read only.
+ *   g_dtype   : DLM_G_F32 (fp32) or DLM_G_BF16 (bfloat16 bit patterns, widened exactly).
+ *   beta      : momentum coefficient in [0, 1)  (Algorithms 1-2 state (0,1); 0 gives DSGD).
+ *   gamma     : learning rate, finite and > 0.
+ * Every output depends on iteration-k inputs only (all nodes update simultaneously, as
+ * the "every node i" loops of Algorithms 1 and 2 prescribe), although x and m are
+ * overwritten.  All arithmetic is fp32.  Traffic: x, m, g read once, x, m written once.
+ * Fastest path: x, m, g 16-byte aligned, ld and ldg multiples of 4 (8 for bf16 g).  Other
+ * layouts take a slower scalar path; pointers need only element alignment.
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_HYPER,
+ *         DLM_ERR_KIND, DLM_ERR_UNSUPPORTED, DLM_ERR_CUDA.
+ * ------------------------------------------------------------------------------------ */
+enum { DLM_G_F32 = 0, DLM_G_BF16 = 1 };
+
+/*
+ * DecentLaM (Sec. 5, Eqs. decentLaM-x-1..3; Algorithm 2).  With W = topo slot:
+ *   g~_i = sum_{j in N_i} w_ij g_j + (1/gamma) sum_{j in N_i, j != i} w_ij (x_i - x_j)
+ *   m_i <- beta m_i + g~_i ;   x_i <- x_i - gamma m_i(new)
+ * which is g~ = W g + (1/gamma)(I - W) x with (I - W) having an exactly zero row sum; for
+ * a W with unit row sums it equals the per-node expression of Eq. (DecentLaM-gi).
+ */
+int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
+                   float* x, float* m, const void* g, int g_dtype, int64_t ldg,
+                   float beta, float gamma, void* cuda_stream);
+
+/*
+ * DmSGD (Algorithm 1; App. A matrix form):
+ *   m_i <- beta m_i + g_i ;  y_i = x_i - gamma m_i(new) ;
+ *   x_i <- y_i + sum_{j in N_i, j != i} w_ij (y_j - y_i)      (= sum_j w_ij y_j for unit row sums)
+ */
+int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
+               float* x, float* m, const void* g, int g_dtype, int64_t ldg,
+               float beta, float gamma, void* cuda_stream);
+
+/*
+ * Parallel momentum SGD on the globally averaged gradient (Sec. 1, Sec. 7 "PmSGD"):
+ *   gbar = (1/n) sum_i g_i ;  m_i <- beta m_i + gbar ;  x_i <- x_i - gamma m_i(new)
+ * No topology: the global average plays the role of W = (1/n) 1 1^T.
+ */
+int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype,
+               int64_t ldg, float beta, float gamma, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------
+ * Full-batch least-squares gradient of the linear-regression experiment (App. G):
+ *   f_i(x) = (scale/2) ||A_i x - b_i||^2 ,   g_i = scale * A_i^T (A_i x_i - b_i).
+ *   A : device fp32 [n, p, q] row-major, 16-byte aligned, q a multiple of 4
+ *   b : device fp32 [n, p];  x : device fp32 [n, q] (row stride q);  g : device fp32 [n, q], written
+ *   workspace, workspace_bytes : device scratch of at least lsq_grad_workspace_bytes(n,p,q)
+ *       bytes, 256-byte aligned, owned by the caller; its contents are overwritten and carry
+ *       nothing between calls.  Two calls sharing a workspace must not overlap on the GPU.
+ * A is read exactly once per call.  Partial sums are combined in a fixed order, so repeated
+ * calls give bitwise identical results.
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_UNSUPPORTED
+ *         (q not a multiple of 4 or above 8192), DLM_ERR_WORKSPACE, DLM_ERR_CUDA.
+ * ------------------------------------------------------------------------------------ */
+int64_t lsq_grad_workspace_bytes(int n, int p, int q); /* negative dlm_status on bad sizes */
+
+int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
+             float scale, void* workspace, int64_t workspace_bytes, void* cuda_stream);
+
+/* Kernel launches issued by this library in the calling process so far (all entry points). */
+int64_t dlm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DECENTLAM_H_ */
