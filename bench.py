@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the fused DecentLaM step (node-params updated per second, HBM roofline fraction).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfgX]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: slot selection
+from the topology tables, neighbour mix, momentum update and in-place parameter write of every
+node, i.e. one decentlam_step call on the stacked [n, d] state.  At N = 1 the workload is cfg2
+(n = 16 nodes, d = 25,557,032, one-peer exponential graph).  For N > 1 every rank runs an
+independent replica of the same workload on its own GPU (the path has no exchange step between
+GPUs); the job value is the sum of units over ranks divided by the slowest rank's time.
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decentlam_step_node_params_per_s"
+UNIT = "node-params/s"
+MAX_STEPS_PER_CHUNK = 256   # state is re-initialised (untimed) between chunks: on the directed
+                            # exponential graphs DecentLaM's disagreement modes grow geometrically
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the DmSGD / PmSGD side timings")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.split(",") for r in open(self.path).read().strip().splitlines() if r.strip()]
+            os.unlink(self.path)
+            sm, reasons, mx = [], set(), None
+            for r in rows:
+                r = [c.strip() for c in r]
+                if len(r) < 9:
+                    continue
+                sm.append(float(r[1])); mx = float(r[2])
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            if sm:
+                sm.sort()
+                out = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        except Exception:
+            pass
+        return out
+
+
+def dist_setup(n_gpus):
+    """Returns (rank, world, local_rank, dist or None)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        import torch
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend=backend)
+        return rank, world, local, dist
+    return rank, world, local, None
+
+
+def aggregate_over_ranks(dist, seconds, units, device):
+    """Job-level figures from per-rank ones: slowest rank's time, sum of units (replicas)."""
+    if dist is None:
+        return seconds, units
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def oracle_sample(workload, budget_s=20.0):
+    """Time the CPU oracle's DecentLaM step, as it stands, on a column slab of the workload."""
+    import numpy as np
+
+    import oracle
+    from paper_2104_11981_b200 import inputs
+    w = inputs.WORKLOADS[workload]
+    kinds = {"ring": oracle.RING, "static_exp": oracle.STATIC_EXP, "one_peer_exp": oracle.ONE_PEER_EXP}
+    adj = None
+    if w.topology == "er_mh":
+        adj, _ = inputs.er_adjacency(w.n, w.er_p, inputs.seed_for(workload, inputs.P_GRAPH))
+        kind = oracle.ADJ_MH
+    else:
+        kind = kinds[w.topology]
+    period = oracle.topology_period(kind, w.n)
+    Ws = [oracle.topology_dense(kind, w.n, s, adj) for s in range(period)]
+    cols = min(w.d, (1 << 20) if w.n <= 64 else (1 << 16))
+    threads = os.cpu_count() or 1
+    x = inputs.normal_np((w.n, cols), w.x0_std or 0.02, 1).astype(np.float64)
+    m = np.zeros_like(x)
+    g = inputs.normal_np((w.n, cols), w.g_std or 1e-3, 2).astype(np.float64)
+    times = []
+    t_begin = time.perf_counter()
+    k = 0
+    while k < 3 or (time.perf_counter() - t_begin < budget_s and k < 50):
+        t0 = time.perf_counter()
+        x, m = oracle.decentlam_step(Ws[k % period], x, m, g, np.float32(w.beta), np.float32(w.gamma), threads)
+        times.append(time.perf_counter() - t0)
+        k += 1
+    times.sort()
+    med = times[len(times) // 2]
+    return {"value": w.n * cols / med, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{workload}: {len(times)} DecentLaM steps of the double-precision dense-W oracle on a "
+                      f"[{w.n} x {cols}] column slab (median), {threads} threads"}, med, w.n * cols
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import build as oracle_build
+    oracle_build.build()
+    from paper_2104_11981_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    # each "step" is one oracle step on the bounded slab; warmup + steps of them
+    base, med, units = oracle_sample(args.workload, budget_s=min(60.0, 2.0 * (args.steps + args.warmup)))
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": med * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "n": w.n, "d": w.d, "topology": w.topology,
+                       "note": "CPU oracle on host cores; each step is a bounded column slab"},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def time_steps(step_fn, reset_fn, steps, warmup, torch, stream, count_fn=lambda: 0):
+    """Warm up, then time exactly `steps` calls with CUDA events on `stream` (chunked so the
+    state can be re-initialised, untimed, between chunks).  Returns (seconds, kernel launches
+    of the library inside the timed regions)."""
+    reset_fn()
+    k = 0
+    for _ in range(warmup):
+        step_fn(k); k += 1
+    torch.cuda.synchronize()
+    total_ms, done, launches = 0.0, 0, 0
+    while done < steps:
+        chunk = min(MAX_STEPS_PER_CHUNK - (warmup if done == 0 else 0), steps - done)
+        chunk = max(1, chunk)
+        if done > 0:
+            reset_fn(); k = 0
+            torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0 = count_fn()
+        e0.record(stream)
+        for _ in range(chunk):
+            step_fn(k); k += 1
+        e1.record(stream)
+        e1.synchronize()
+        launches += count_fn() - c0
+        total_ms += e0.elapsed_time(e1)
+        done += chunk
+    return total_ms * 1e-3, launches
+
+
+def run_ours(args):
+    import torch
+
+    from paper_2104_11981_b200 import binding as B   # fails loudly if the CUDA library is missing
+    from paper_2104_11981_b200 import inputs
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    args.warmup = max(args.warmup, 3)
+    rank, world, local, dist = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w = inputs.WORKLOADS[args.workload]
+    if w.p:
+        raise SystemExit("bench.py times the step workloads (cfg1, cfg2, cfg3, cfg5)")
+    n, d = w.n, w.d
+    gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+
+    if w.topology == "er_mh":
+        adj, _ = inputs.er_adjacency(n, w.er_p, inputs.seed_for(args.workload, inputs.P_GRAPH))
+        rowptr, col = inputs.adjacency_to_lists(adj)
+        topo = B.topology_build(B.CSR_MH, n, rowptr, col)
+    else:
+        topo = B.topology_build({"ring": B.RING, "static_exp": B.STATIC_EXP, "one_peer_exp": B.ONE_PEER_EXP}[w.topology], n)
+
+    x0 = inputs.normal_torch((n, d), w.x0_std, inputs.seed_for(args.workload, inputs.P_X0) + rank, dev)
+    x = torch.empty_like(x0); m = torch.empty_like(x0)
+    g = inputs.normal_torch((n, d), w.g_std, inputs.seed_for(args.workload, inputs.P_G0) + rank, dev, dtype=gdt)
+    stream = torch.cuda.current_stream()
+
+    def reset():
+        x.copy_(x0); m.zero_()
+
+    def decentlam(k):
+        B.decentlam_step(topo, k, x, m, g, w.beta, w.gamma)
+
+    bytes_per_np = 16 + g.element_size()          # x, m read + x, m written + g read
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    secs, launches = time_steps(decentlam, reset, args.steps, args.warmup, torch, stream, B.launch_count)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if dist is not None:
+        dist.barrier()
+    err = B.kernel_error()
+    if err:
+        raise SystemExit(f"bench.py: step kernel reported error {err}")
+    job_secs, job_units = aggregate_over_ranks(dist, secs, n * d * args.steps, dev)
+    value = job_units / job_secs
+    peak, peak_kind = measured_peak()
+    achieved = bytes_per_np * n * d * args.steps / secs / 1e9
+
+    extra = {}
+    if not args.no_extra and world == 1:
+        for name, fn in (("dmsgd", lambda k: B.dmsgd_step(topo, k, x, m, g, w.beta, w.gamma)),
+                         ("pmsgd", lambda k: B.pmsgd_step(x, m, g, w.beta, w.gamma))):
+            steps_x = max(10, args.steps // 2)
+            s, _ = time_steps(fn, reset, steps_x, 3, torch, stream)
+            extra[name] = {"ms_per_step": s / steps_x * 1e3, "value": n * d * steps_x / s,
+                           "gbs": bytes_per_np * n * d * steps_x / s / 1e9}
+
+    e2e = None
+    if not args.no_e2e:
+        # End to end: this step's gradients arrive from pinned host memory, the step runs, and a
+        # slice of the updated parameters is read back.  x and m stay resident (they are state).
+        g_host = torch.empty((n, d), dtype=gdt, pin_memory=True)
+        g_host.copy_(g)
+        g_dev = torch.empty_like(g)
+        cols_back = min(d, 4096)
+        res_host = torch.empty((n, cols_back), dtype=torch.float32, pin_memory=True)
+        e_steps = max(3, min(args.steps, 10))
+        reset()
+        for k in range(2):
+            g_dev.copy_(g_host, non_blocking=True); B.decentlam_step(topo, k, x, m, g_dev, w.beta, w.gamma)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for k in range(e_steps):
+            g_dev.copy_(g_host, non_blocking=True)
+            B.decentlam_step(topo, k, x, m, g_dev, w.beta, w.gamma)
+            res_host.copy_(x[:, :cols_back], non_blocking=True)
+        e1.record(stream)
+        e1.synchronize()
+        e_secs = e0.elapsed_time(e1) * 1e-3
+        je_secs, je_units = aggregate_over_ranks(dist, e_secs, n * d * e_steps, dev)
+        e2e = {"value": je_units / je_secs, "unit": UNIT, "h2d_bytes_per_step": n * d * g.element_size(),
+               "d2h_bytes_per_step": n * cols_back * 4, "steps": e_steps,
+               "note": "gradients copied from pinned host memory every step; x, m resident"}
+        del g_host, g_dev
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import build as oracle_build
+        oracle_build.build()
+        cpu_baseline, _, _ = oracle_sample(args.workload)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
+                       "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       "l2": f"working set {(8 + g.element_size()) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": f"of {peak_kind}",
+                         "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d},
+            "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "other_rules": extra,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

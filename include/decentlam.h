@@ -21,6 +21,12 @@
 
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define DLM_API __attribute__((visibility("default")))
+#else
+#define DLM_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -40,7 +46,7 @@ typedef enum dlm_status {
 } dlm_status;
 
 /* Human-readable name of a status code; never NULL. */
-const char* dlm_status_string(int status);
+DLM_API const char* dlm_status_string(int status);
 
 /* ------------------------------------------------------------------------------------
  * Topology: the weight matrix W = [w_ij] of Sec. 3 ("Network topology and weights"),
@@ -78,28 +84,30 @@ typedef enum dlm_topology_kind {
  *                          sum within 1e-6 of 1 (doubly stochastic, Assumption A.3).
  *   out : receives the handle.  The library owns it (host and device tables) until
  *         topology_destroy.  The inputs are copied; the caller may free them at once.
+ *         In a process without a CUDA device the handle is host-only: the host tables can
+ *         be read, topology_tables_device returns NULL pointers and steps fail with DLM_ERR_CUDA.
  * Errors: DLM_ERR_NULL, DLM_ERR_KIND, DLM_ERR_SHAPE (n too small for the kind),
  *         DLM_ERR_UNSUPPORTED (n > DLM_MAX_NODES), DLM_ERR_TOPOLOGY, DLM_ERR_CUDA.
  */
-int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
+DLM_API int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
                    dlm_topology** out);
 
 /* Number of distinct slots; iteration k uses slot k mod period (k = 0 is the first step). */
-int topology_period(const dlm_topology* topo, int* period);
+DLM_API int topology_period(const dlm_topology* topo, int* period);
 
 /* Number of nodes the topology was built for. */
-int topology_nodes(const dlm_topology* topo, int* n);
+DLM_API int topology_nodes(const dlm_topology* topo, int* n);
 
 /* Borrowed pointers to the CSR tables of one slot, valid until topology_destroy.
  * _host returns host pointers, _device device pointers.  Any out-pointer may be NULL.
  * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE (slot outside [0, period)). */
-int topology_tables_host(const dlm_topology* topo, int slot, const int32_t** rowptr,
+DLM_API int topology_tables_host(const dlm_topology* topo, int slot, const int32_t** rowptr,
                          const int32_t** col, const float** val, int64_t* nnz);
-int topology_tables_device(const dlm_topology* topo, int slot, const int32_t** rowptr,
+DLM_API int topology_tables_device(const dlm_topology* topo, int slot, const int32_t** rowptr,
                            const int32_t** col, const float** val, int64_t* nnz);
 
 /* Free host and device tables.  NULL is accepted. */
-int topology_destroy(dlm_topology* topo);
+DLM_API int topology_destroy(dlm_topology* topo);
 
 /* ------------------------------------------------------------------------------------
  * Update rules.  Common arguments:
@@ -128,7 +136,7 @@ enum { DLM_G_F32 = 0, DLM_G_BF16 = 1 };
  * which is g~ = W g + (1/gamma)(I - W) x with (I - W) having an exactly zero row sum; for
  * a W with unit row sums it equals the per-node expression of Eq. (DecentLaM-gi).
  */
-int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
+DLM_API int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
                    float* x, float* m, const void* g, int g_dtype, int64_t ldg,
                    float beta, float gamma, void* cuda_stream);
 
@@ -137,7 +145,7 @@ int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_
  *   m_i <- beta m_i + g_i ;  y_i = x_i - gamma m_i(new) ;
  *   x_i <- y_i + sum_{j in N_i, j != i} w_ij (y_j - y_i)      (= sum_j w_ij y_j for unit row sums)
  */
-int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
+DLM_API int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
                float* x, float* m, const void* g, int g_dtype, int64_t ldg,
                float beta, float gamma, void* cuda_stream);
 
@@ -146,29 +154,49 @@ int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld
  *   gbar = (1/n) sum_i g_i ;  m_i <- beta m_i + gbar ;  x_i <- x_i - gamma m_i(new)
  * No topology: the global average plays the role of W = (1/n) 1 1^T.
  */
-int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype,
+DLM_API int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype,
                int64_t ldg, float beta, float gamma, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------
  * Full-batch least-squares gradient of the linear-regression experiment (App. G):
  *   f_i(x) = (scale/2) ||A_i x - b_i||^2 ,   g_i = scale * A_i^T (A_i x_i - b_i).
- *   A : device fp32 [n, p, q] row-major, 16-byte aligned, q a multiple of 4
- *   b : device fp32 [n, p];  x : device fp32 [n, q] (row stride q);  g : device fp32 [n, q], written
+ *   A : device fp32 [n, p, q] row-major, 16-byte aligned; 1 <= q <= 8192
+ *   b : device fp32 [n, p];  x : device fp32 [n, q] (row stride q), 16-byte aligned;
+ *   g : device fp32 [n, q], 16-byte aligned, written
  *   workspace, workspace_bytes : device scratch of at least lsq_grad_workspace_bytes(n,p,q)
  *       bytes, 256-byte aligned, owned by the caller; its contents are overwritten and carry
  *       nothing between calls.  Two calls sharing a workspace must not overlap on the GPU.
- * A is read exactly once per call.  Partial sums are combined in a fixed order, so repeated
- * calls give bitwise identical results.
+ * Fast path (A read from HBM exactly once): q a multiple of 128 and at most 1024; other q use a
+ * kernel that re-reads each 8-row block from cache.  Partial sums are combined in a fixed
+ * order, so repeated calls give bitwise identical results.
  * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_UNSUPPORTED
- *         (q not a multiple of 4 or above 8192), DLM_ERR_WORKSPACE, DLM_ERR_CUDA.
+ *         (q above 8192), DLM_ERR_WORKSPACE, DLM_ERR_CUDA.
  * ------------------------------------------------------------------------------------ */
-int64_t lsq_grad_workspace_bytes(int n, int p, int q); /* negative dlm_status on bad sizes */
+DLM_API int64_t lsq_grad_workspace_bytes(int n, int p, int q); /* negative dlm_status on bad sizes */
 
-int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
+DLM_API int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
              float scale, void* workspace, int64_t workspace_bytes, void* cuda_stream);
 
 /* Kernel launches issued by this library in the calling process so far (all entry points). */
-int64_t dlm_launch_count(void);
+DLM_API int64_t dlm_launch_count(void);
+
+/*
+ * The pipelined step kernel bounds every wait on its copy barriers; if a wait ever runs out the
+ * kernel records a non-zero code, stops early and the step's output is incomplete.  This call
+ * synchronises with the device, returns the recorded code in *flag (0 = none) and clears it.
+ */
+DLM_API int dlm_kernel_error(int* flag);
+
+/*
+ * Expert performance knobs of the step kernels (process-wide, not thread-safe; 0 = automatic):
+ *   knob 0  kernel path: 1 = plain-load tile kernel, 2 = bulk-copy pipeline kernel (steps whose
+ *           layout cannot use it then return DLM_ERR_UNSUPPORTED)
+ *   knob 1  tile width in columns (power of two)
+ *   knob 2  pipeline stages
+ *   knob 3  CTAs per SM the pipeline kernel sizes its shared memory for
+ * Results do not depend on the knobs (all paths round identically).  DLM_ERR_KIND for an unknown knob.
+ */
+DLM_API int dlm_set_tuning(int knob, int value);
 
 #ifdef __cplusplus
 }

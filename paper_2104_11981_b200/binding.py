@@ -1,0 +1,211 @@
+"""ctypes binding of libdecentlam.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name (include/decentlam.h).  Tensors are
+torch CUDA tensors used purely as device memory; only their data pointers, strides and the
+current stream cross the boundary.  A non-zero status raises DecentlamError.  There is no
+fallback: if the shared library is missing, importing this module fails.
+"""
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdecentlam.so")
+
+RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, CSR_MH, CSR_WEIGHTS = range(6)
+G_F32, G_BF16 = 0, 1
+MAX_NODES = 2048
+
+STATUS = {0: "DLM_OK", -1: "DLM_ERR_NULL", -2: "DLM_ERR_SHAPE", -3: "DLM_ERR_ALIGN", -4: "DLM_ERR_ALIAS",
+          -5: "DLM_ERR_HYPER", -6: "DLM_ERR_KIND", -7: "DLM_ERR_TOPOLOGY", -8: "DLM_ERR_UNSUPPORTED",
+          -9: "DLM_ERR_CUDA", -10: "DLM_ERR_WORKSPACE"}
+
+
+class DecentlamError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        msg = _lib.dlm_status_string(self.status).decode()
+        super().__init__(f"{where}: {STATUS.get(self.status, self.status)} ({msg})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2104_11981_b200.build` "
+                      "(there is no CPU fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+_i32p = ctypes.POINTER(ctypes.c_int32)
+_f32p = ctypes.POINTER(ctypes.c_float)
+_vp = ctypes.c_void_p
+_i64 = ctypes.c_int64
+_int = ctypes.c_int
+_flt = ctypes.c_float
+
+_lib.dlm_status_string.argtypes = [_int]
+_lib.dlm_status_string.restype = ctypes.c_char_p
+_lib.topology_build.argtypes = [_int, _int, _vp, _vp, _vp, ctypes.POINTER(_vp)]
+_lib.topology_period.argtypes = [_vp, ctypes.POINTER(_int)]
+_lib.topology_nodes.argtypes = [_vp, ctypes.POINTER(_int)]
+for _name in ("topology_tables_host", "topology_tables_device"):
+    getattr(_lib, _name).argtypes = [_vp, _int, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                     ctypes.POINTER(_i64)]
+_lib.topology_destroy.argtypes = [_vp]
+for _name in ("decentlam_step", "dmsgd_step"):
+    getattr(_lib, _name).argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
+_lib.pmsgd_step.argtypes = [_int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
+_lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
+_lib.lsq_grad_workspace_bytes.restype = _i64
+_lib.lsq_grad.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp, _i64, _vp]
+_lib.dlm_launch_count.argtypes = []
+_lib.dlm_launch_count.restype = _i64
+_lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
+_lib.dlm_set_tuning.argtypes = [_int, _int]
+
+EXPORTS = ["dlm_status_string", "topology_build", "topology_period", "topology_nodes", "topology_tables_host",
+           "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "pmsgd_step",
+           "lsq_grad_workspace_bytes", "lsq_grad", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise DecentlamError(rc, where)
+
+
+def raw():
+    """The ctypes library object (for tests that pass deliberately bad arguments)."""
+    return _lib
+
+
+class Topology:
+    """Owner of a dlm_topology handle."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def destroy(self):
+        if getattr(self, "handle", None):
+            _lib.topology_destroy(self.handle)
+            self.handle = None
+
+    @property
+    def period(self):
+        v = _int()
+        _check(_lib.topology_period(self.handle, ctypes.byref(v)), "topology_period")
+        return v.value
+
+    @property
+    def n(self):
+        v = _int()
+        _check(_lib.topology_nodes(self.handle, ctypes.byref(v)), "topology_nodes")
+        return v.value
+
+    def tables_host(self, slot=0):
+        """(rowptr int32[n+1], col int32[nnz], val float32[nnz]) copies of one slot's CSR tables."""
+        import numpy as np
+        rp, cp, vp, nnz = _vp(), _vp(), _vp(), _i64()
+        _check(_lib.topology_tables_host(self.handle, slot, ctypes.byref(rp), ctypes.byref(cp), ctypes.byref(vp),
+                                         ctypes.byref(nnz)), "topology_tables_host")
+        n, z = self.n, nnz.value
+        rowptr = np.ctypeslib.as_array(ctypes.cast(rp, _i32p), shape=(n + 1,)).copy()
+        col = np.ctypeslib.as_array(ctypes.cast(cp, _i32p), shape=(z,)).copy()
+        val = np.ctypeslib.as_array(ctypes.cast(vp, _f32p), shape=(z,)).copy()
+        return rowptr, col, val
+
+    def tables_device(self, slot=0):
+        """Raw device addresses (rowptr, col, val) and nnz of one slot."""
+        rp, cp, vp, nnz = _vp(), _vp(), _vp(), _i64()
+        _check(_lib.topology_tables_device(self.handle, slot, ctypes.byref(rp), ctypes.byref(cp), ctypes.byref(vp),
+                                           ctypes.byref(nnz)), "topology_tables_device")
+        return rp.value, cp.value, vp.value, nnz.value
+
+
+def topology_build(kind, n, rowptr=None, col=None, val=None):
+    import numpy as np
+
+    def ptr(a, dt):
+        if a is None:
+            return None, None
+        a = np.ascontiguousarray(a, dtype=dt)
+        return a, a.ctypes.data_as(_vp)
+
+    keep_r, pr = ptr(rowptr, np.int32)
+    keep_c, pc = ptr(col, np.int32)
+    keep_v, pv = ptr(val, np.float32)
+    out = _vp()
+    _check(_lib.topology_build(kind, n, pr, pc, pv, ctypes.byref(out)), "topology_build")
+    return Topology(out)
+
+
+def _stream_ptr(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return _vp(s.cuda_stream)
+
+
+def _state_args(x, m, g):
+    import torch
+    assert x.is_cuda and m.is_cuda and g.is_cuda, "device tensors required"
+    assert x.dtype == torch.float32 and m.dtype == torch.float32
+    assert x.dim() == 2 and m.shape == x.shape and g.shape == x.shape
+    assert x.stride(1) == 1 and m.stride(1) == 1 and g.stride(1) == 1 and m.stride(0) == x.stride(0)
+    if g.dtype == torch.float32:
+        gd = G_F32
+    elif g.dtype == torch.bfloat16:
+        gd = G_BF16
+    else:
+        raise TypeError("g must be float32 or bfloat16")
+    n, d = x.shape
+    return n, d, x.stride(0), _vp(x.data_ptr()), _vp(m.data_ptr()), _vp(g.data_ptr()), gd, g.stride(0)
+
+
+def decentlam_step(topo, k, x, m, g, beta, gamma, stream=None):
+    n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
+    _check(_lib.decentlam_step(topo.handle, k, n, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)),
+           "decentlam_step")
+
+
+def dmsgd_step(topo, k, x, m, g, beta, gamma, stream=None):
+    n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
+    _check(_lib.dmsgd_step(topo.handle, k, n, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)),
+           "dmsgd_step")
+
+
+def pmsgd_step(x, m, g, beta, gamma, stream=None):
+    n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
+    _check(_lib.pmsgd_step(n, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)), "pmsgd_step")
+
+
+def lsq_grad_workspace_bytes(n, p, q):
+    v = _lib.lsq_grad_workspace_bytes(n, p, q)
+    if v < 0:
+        raise DecentlamError(v, "lsq_grad_workspace_bytes")
+    return int(v)
+
+
+def lsq_grad(A, b, x, g, scale, workspace, stream=None):
+    """g <- scale * A_i^T (A_i x_i - b_i).  A [n,p,q], b [n,p], x [n,q], g [n,q] contiguous fp32 device
+    tensors; workspace: uint8 device tensor of at least lsq_grad_workspace_bytes(n, p, q) bytes."""
+    n, p, q = A.shape
+    assert A.is_contiguous() and b.is_contiguous() and x.is_contiguous() and g.is_contiguous()
+    assert b.shape == (n, p) and x.shape == (n, q) and g.shape == (n, q)
+    _check(_lib.lsq_grad(n, p, q, _vp(A.data_ptr()), _vp(b.data_ptr()), _vp(x.data_ptr()), _vp(g.data_ptr()),
+                         scale, _vp(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
+                         _stream_ptr(stream)), "lsq_grad")
+
+
+def launch_count():
+    return int(_lib.dlm_launch_count())
+
+
+def kernel_error():
+    v = _int()
+    _check(_lib.dlm_kernel_error(ctypes.byref(v)), "dlm_kernel_error")
+    return v.value
+
+
+def set_tuning(knob, value):
+    _check(_lib.dlm_set_tuning(knob, value), "dlm_set_tuning")

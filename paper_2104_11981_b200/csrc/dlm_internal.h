@@ -1,0 +1,51 @@
+// Internal declarations shared by the translation units of libdecentlam (not installed).
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "decentlam.h"
+
+// One time slot of a topology: CSR on the host and its copy on the device.
+struct dlm_slot {
+    std::vector<int32_t> rowptr, col;
+    std::vector<float> val;
+    int32_t* d_rowptr = nullptr;
+    int32_t* d_col = nullptr;
+    float* d_val = nullptr;
+    int max_degree = 0;  // longest row, self included
+};
+
+struct dlm_topology {
+    int n = 0;
+    int kind = 0;
+    int device = -1;  // CUDA device holding the tables
+    std::vector<dlm_slot> slots;
+};
+
+enum dlm_rule { DLM_RULE_DECENTLAM = 0, DLM_RULE_DMSGD = 1 };
+
+// Arguments of one fused step over the columns [0, d) of row-major [n, ld] arrays.
+struct dlm_step_args {
+    int n;
+    int64_t d, ld, ldg;
+    float* x;
+    float* m;
+    const void* g;
+    int g_dtype;
+    const int32_t* rowptr;  // device
+    const int32_t* col;     // device
+    const float* val;       // device
+    int nnz;
+    int max_degree;
+    float beta, gamma, inv_gamma;
+};
+
+// Launchers (step_kernels.cu, pmsgd_kernel.cu, lsq_kernels.cu).  Return a dlm_status.
+int dlm_launch_step(int rule, const dlm_step_args& a, void* stream);
+int dlm_launch_pmsgd(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype,
+                     int64_t ldg, float beta, float gamma, void* stream);
+int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
+                        float scale, float* partial, void* stream);
+int dlm_lsq_splits(int n, int p, int q);  // row chunks per node used by lsq_grad
+
+void dlm_count_launch(int launches);

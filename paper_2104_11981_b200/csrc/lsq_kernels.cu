@@ -1,0 +1,192 @@
+// Full-batch least-squares gradient of the linear-regression experiment (App. G):
+//   g_i = scale * A_i^T (A_i x_i - b_i),   A [n, p, q] row-major.
+// A is streamed from HBM exactly once.  A warp owns whole rows of A_i: it forms the residual
+// r_a = <A_i[a,:], x_i> - b_i[a] with a butterfly reduction and at once adds r_a * A_i[a,:] to
+// its per-lane slice of A_i^T r, using the row values still held in registers.  Each node's
+// rows are split over S CTAs; warp partials are summed inside the CTA, CTA partials go to
+// scratch [n, S, q] and a second tiny kernel adds them in a fixed order (bitwise repeatable).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+
+#include "dlm_internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxSplits = 64;
+
+__device__ __forceinline__ float warp_allsum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// q == 128 * Q4: lane l holds the float4 groups l, l+32, ..., of a row (coalesced 512-byte pieces).
+template <int Q4>
+__global__ void __launch_bounds__(kThreads) lsq_partial_rows_kernel(int p, int q, int rows_per_split, int splits,
+                                                                     const float* __restrict__ A,
+                                                                     const float* __restrict__ b,
+                                                                     const float* __restrict__ x,
+                                                                     float* __restrict__ partial) {
+    __shared__ __align__(16) float red[kWarps][128 * Q4];
+    const int s = blockIdx.x, i = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = s * rows_per_split, r1 = min(p, r0 + rows_per_split);
+    const float4* Ai = reinterpret_cast<const float4*>(A + (size_t)i * p * q);
+    const float4* xi = reinterpret_cast<const float4*>(x + (size_t)i * q);
+    const float* bi = b + (size_t)i * p;
+    const int q4 = q >> 2;
+
+    float4 xr[Q4], acc[Q4], cur[Q4], nxt[Q4];
+#pragma unroll
+    for (int t = 0; t < Q4; ++t) {
+        xr[t] = xi[lane + 32 * t];
+        acc[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    int r = r0 + warp;
+    if (r < r1) {
+#pragma unroll
+        for (int t = 0; t < Q4; ++t) cur[t] = __ldcs(Ai + (size_t)r * q4 + lane + 32 * t);
+    }
+    for (; r < r1; r += kWarps) {
+        const int rn = r + kWarps;
+        if (rn < r1) {
+#pragma unroll
+            for (int t = 0; t < Q4; ++t) nxt[t] = __ldcs(Ai + (size_t)rn * q4 + lane + 32 * t);
+        }
+        float dot = 0.f;
+#pragma unroll
+        for (int t = 0; t < Q4; ++t) {
+            dot = fmaf(cur[t].x, xr[t].x, dot);
+            dot = fmaf(cur[t].y, xr[t].y, dot);
+            dot = fmaf(cur[t].z, xr[t].z, dot);
+            dot = fmaf(cur[t].w, xr[t].w, dot);
+        }
+        const float res = warp_allsum(dot) - bi[r];
+#pragma unroll
+        for (int t = 0; t < Q4; ++t) {
+            acc[t].x = fmaf(cur[t].x, res, acc[t].x);
+            acc[t].y = fmaf(cur[t].y, res, acc[t].y);
+            acc[t].z = fmaf(cur[t].z, res, acc[t].z);
+            acc[t].w = fmaf(cur[t].w, res, acc[t].w);
+        }
+#pragma unroll
+        for (int t = 0; t < Q4; ++t) cur[t] = nxt[t];
+    }
+#pragma unroll
+    for (int t = 0; t < Q4; ++t) reinterpret_cast<float4*>(red[warp])[lane + 32 * t] = acc[t];
+    __syncthreads();
+    float* out = partial + ((size_t)i * splits + s) * q;
+    for (int c = threadIdx.x; c < q; c += kThreads) {
+        float v = red[0][c];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) v += red[w][c];
+        out[c] = v;
+    }
+}
+
+// Any q <= 8192: a CTA takes 8 rows at a time (one per warp) for the residuals, then every thread
+// adds the 8 rank-one contributions to its own columns (second read of the rows comes from cache).
+constexpr int kGenericMaxQ = 8192;
+__global__ void __launch_bounds__(kThreads) lsq_partial_generic_kernel(int p, int q, int rows_per_split, int splits,
+                                                                        const float* __restrict__ A,
+                                                                        const float* __restrict__ b,
+                                                                        const float* __restrict__ x,
+                                                                        float* __restrict__ partial) {
+    __shared__ float res[kWarps];
+    const int s = blockIdx.x, i = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = s * rows_per_split, r1 = min(p, r0 + rows_per_split);
+    const float* Ai = A + (size_t)i * p * q;
+    const float* xi = x + (size_t)i * q;
+    const float* bi = b + (size_t)i * p;
+    float acc[kGenericMaxQ / kThreads];
+#pragma unroll
+    for (int t = 0; t < kGenericMaxQ / kThreads; ++t) acc[t] = 0.f;
+    for (int rb = r0; rb < r1; rb += kWarps) {
+        const int r = rb + warp;
+        float dot = 0.f;
+        if (r < r1)
+            for (int c = lane; c < q; c += 32) dot = fmaf(Ai[(size_t)r * q + c], xi[c], dot);
+        dot = warp_allsum(dot);
+        __syncthreads();
+        if (lane == 0) res[warp] = (r < r1) ? dot - bi[r] : 0.f;
+        __syncthreads();
+        const int rows = min(kWarps, r1 - rb);
+#pragma unroll
+        for (int t = 0; t < kGenericMaxQ / kThreads; ++t) {
+            const int c = threadIdx.x + t * kThreads;
+            if (c < q)
+                for (int w = 0; w < rows; ++w) acc[t] = fmaf(Ai[(size_t)(rb + w) * q + c], res[w], acc[t]);
+        }
+    }
+    float* out = partial + ((size_t)i * splits + s) * q;
+#pragma unroll
+    for (int t = 0; t < kGenericMaxQ / kThreads; ++t) {
+        const int c = threadIdx.x + t * kThreads;
+        if (c < q) out[c] = acc[t];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) lsq_reduce_kernel(int n, int q, int splits, float scale,
+                                                               const float* __restrict__ partial,
+                                                               float* __restrict__ g) {
+    const long long e = (long long)blockIdx.x * kThreads + threadIdx.x;
+    if (e >= (long long)n * q) return;
+    const int i = (int)(e / q), c = (int)(e % q);
+    const float* src = partial + (size_t)i * splits * q + c;
+    float v = src[0];
+    for (int s = 1; s < splits; ++s) v += src[(size_t)s * q];
+    g[e] = scale * v;
+}
+
+}  // namespace
+
+int dlm_lsq_max_splits() { return kMaxSplits; }
+
+int dlm_lsq_splits(int n, int p, int q) {
+    (void)q;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return -1;
+    // one wave of CTAs (two resident per SM): S row chunks per node, each a multiple of 8 rows
+    int S = std::max(1, (2 * sms) / n);
+    S = std::min(S, kMaxSplits);
+    S = std::min(S, std::max(1, p / (4 * kWarps)));
+    int rows = ((p + S - 1) / S + kWarps - 1) / kWarps * kWarps;
+    return (p + rows - 1) / rows;
+}
+
+int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
+                        float scale, float* partial, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int S = dlm_lsq_splits(n, p, q);
+    if (S < 1) return DLM_ERR_CUDA;
+    int rows = ((p + S - 1) / S + kWarps - 1) / kWarps * kWarps;
+    dim3 grid((unsigned)S, (unsigned)n);
+    const bool fast = (q % 128 == 0) && q <= 1024;
+    if (fast) {
+        switch (q / 128) {
+        case 1: lsq_partial_rows_kernel<1><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 2: lsq_partial_rows_kernel<2><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 3: lsq_partial_rows_kernel<3><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 4: lsq_partial_rows_kernel<4><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 5: lsq_partial_rows_kernel<5><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 6: lsq_partial_rows_kernel<6><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        case 7: lsq_partial_rows_kernel<7><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        default: lsq_partial_rows_kernel<8><<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial); break;
+        }
+    } else {
+        if (q > kGenericMaxQ) return DLM_ERR_UNSUPPORTED;
+        lsq_partial_generic_kernel<<<grid, kThreads, 0, st>>>(p, q, rows, S, A, b, x, partial);
+    }
+    if (cudaGetLastError() != cudaSuccess) return DLM_ERR_CUDA;
+    long long total = (long long)n * q;
+    lsq_reduce_kernel<<<(unsigned)((total + kThreads - 1) / kThreads), kThreads, 0, st>>>(n, q, S, scale, partial, g);
+    dlm_count_launch(2);
+    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}

@@ -1,0 +1,614 @@
+// Fused DecentLaM / DmSGD iteration kernels for sm_100a.
+//
+// Data dependence: every rule is coordinate-wise (Eq. DecentLaM-gi acts on each coordinate of
+// x_j, g_j separately), nodes are coupled only through the weights.  A CTA therefore owns a
+// column tile [n x C] of ALL n rows: it stages the iteration-k values of the tile on chip,
+// and only then writes x and m of the same tile.  This makes the in-place update exact
+// (simultaneous update of all nodes) with each of x, m, g read once and x, m written once.
+//
+// Two implementations of the same arithmetic:
+//   step_tma_kernel   persistent CTAs, multi-stage pipeline of 2-D tensor bulk copies
+//                     (cp.async.bulk.tensor) completing on mbarriers; needs 16-byte aligned rows.
+//   step_tile_kernel  plain vector/scalar loads into shared memory; any alignment, any n,
+//                     also used for the last d mod 4 columns.
+// Both call the same per-element update functions, so their results are bitwise identical.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <mutex>
+
+#include "dlm_internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kWaitLimit = 1u << 22;  // polls before a pipeline wait gives up
+
+__device__ int g_kernel_error = 0;  // set to a non-zero code if a bounded wait ran out
+
+// ---------------------------------------------------------------------------------------------
+// Per-element arithmetic (fp32, explicit FMAs so every kernel variant rounds identically).
+// ---------------------------------------------------------------------------------------------
+// DecentLaM (Eqs. decentLaM-x-1..3):  g~ = (W g)_i + ((I - W) x)_i / gamma ; m' = beta m + g~ ; x' = x - gamma m'
+__device__ __forceinline__ void decentlam_finish(float mixg, float cons, float xi, float mi, float beta,
+                                                 float gamma, float inv_gamma, float& mn, float& xn) {
+    float gt = fmaf(cons, inv_gamma, mixg);
+    mn = fmaf(beta, mi, gt);
+    xn = fmaf(-gamma, mn, xi);
+}
+// DmSGD (Algorithm 1), local half:  m' = beta m + g ; y = x - gamma m'
+__device__ __forceinline__ void dmsgd_local(float xi, float mi, float gi, float beta, float gamma, float& mn,
+                                            float& y) {
+    mn = fmaf(beta, mi, gi);
+    y = fmaf(-gamma, mn, xi);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
+
+template <int VEC>
+struct Pack {
+    float v[VEC];
+};
+
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_f32(const float* p);
+template <>
+__device__ __forceinline__ Pack<4> ld_f32<4>(const float* p) {
+    float4 t = *reinterpret_cast<const float4*>(p);
+    return {{t.x, t.y, t.z, t.w}};
+}
+template <>
+__device__ __forceinline__ Pack<1> ld_f32<1>(const float* p) {
+    return {{*p}};
+}
+template <int VEC>
+__device__ __forceinline__ void st_f32(float* p, const Pack<VEC>& a);
+template <>
+__device__ __forceinline__ void st_f32<4>(float* p, const Pack<4>& a) {
+    *reinterpret_cast<float4*>(p) = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
+}
+template <>
+__device__ __forceinline__ void st_f32<1>(float* p, const Pack<1>& a) {
+    *p = a.v[0];
+}
+// gradient loads: fp32 or bf16 bit patterns widened exactly
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_g(const float* p) {
+    return ld_f32<VEC>(p);
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_g(const __nv_bfloat16* p);
+template <>
+__device__ __forceinline__ Pack<4> ld_g<4>(const __nv_bfloat16* p) {
+    uint2 u = *reinterpret_cast<const uint2*>(p);
+    return {{__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+             __uint_as_float(u.y & 0xffff0000u)}};
+}
+template <>
+__device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
+    return {{bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(p))}};
+}
+
+// Neighbour tables of the current slot, either copied to shared memory or left in global memory.
+struct Tables {
+    const int* rowptr;
+    const int* col;
+    const float* val;
+};
+
+__device__ __forceinline__ Tables stage_tables(const dlm_step_args& a, void* smem_tables, bool in_smem) {
+    if (!in_smem) return {a.rowptr, a.col, a.val};
+    int* s_rowptr = reinterpret_cast<int*>(smem_tables);
+    int* s_col = s_rowptr + (a.n + 1);
+    float* s_val = reinterpret_cast<float*>(s_col + a.nnz);
+    for (int i = threadIdx.x; i <= a.n; i += blockDim.x) s_rowptr[i] = a.rowptr[i];
+    for (int i = threadIdx.x; i < a.nnz; i += blockDim.x) {
+        s_col[i] = a.col[i];
+        s_val[i] = a.val[i];
+    }
+    return {s_rowptr, s_col, s_val};
+}
+
+// Mix one item (row i, VEC consecutive columns at tile offset off) of the DecentLaM rule.
+//   xs, gs: staged tiles [n][C] (gs may hold bf16 when GS is __nv_bfloat16)
+template <int VEC, typename GS>
+__device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, int C, const float* xs,
+                                               const GS* gs, const Pack<VEC>& mi, float beta, float gamma,
+                                               float inv_gamma, Pack<VEC>& mn, Pack<VEC>& xn) {
+    const Pack<VEC> xi = ld_f32<VEC>(xs + (size_t)i * C + off);
+    float mixg[VEC], cons[VEC];
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) mixg[u] = cons[u] = 0.0f;
+    const int p1 = t.rowptr[i + 1];
+    for (int p = t.rowptr[i]; p < p1; ++p) {
+        const int j = t.col[p];
+        const float w = t.val[p];
+        const Pack<VEC> gj = ld_g<VEC>(gs + (size_t)j * C + off);
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
+        if (j != i) {
+            const Pack<VEC> xj = ld_f32<VEC>(xs + (size_t)j * C + off);
+#pragma unroll
+            for (int u = 0; u < VEC; ++u) cons[u] = fmaf(w, xi.v[u] - xj.v[u], cons[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < VEC; ++u)
+        decentlam_finish(mixg[u], cons[u], xi.v[u], mi.v[u], beta, gamma, inv_gamma, mn.v[u], xn.v[u]);
+}
+
+// Partial average of the DmSGD rule on staged y = x - gamma m':  x' = y_i + sum_{j != i} w_ij (y_j - y_i)
+template <int VEC>
+__device__ __forceinline__ void dmsgd_item(const Tables& t, int i, int off, int C, const float* ys,
+                                           Pack<VEC>& xn) {
+    const Pack<VEC> yi = ld_f32<VEC>(ys + (size_t)i * C + off);
+    float acc[VEC];
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) acc[u] = 0.0f;
+    const int p1 = t.rowptr[i + 1];
+    for (int p = t.rowptr[i]; p < p1; ++p) {
+        const int j = t.col[p];
+        if (j == i) continue;
+        const float w = t.val[p];
+        const Pack<VEC> yj = ld_f32<VEC>(ys + (size_t)j * C + off);
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) acc[u] = fmaf(w, yj.v[u] - yi.v[u], acc[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) xn.v[u] = yi.v[u] + acc[u];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Plain-load tile kernel (any alignment).  C is a power of two multiple of VEC.
+// Shared memory: xs[n*C] fp32 (x, or y for DmSGD) | gs[n*C] fp32 (DecentLaM only) | tables.
+// ---------------------------------------------------------------------------------------------
+template <int RULE, typename GT, int VEC>
+__global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, int C, int cv_shift,
+                                                              int tables_in_smem, long long num_tiles) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* xs = reinterpret_cast<float*>(smem_raw);
+    float* gs = xs + (size_t)a.n * C;
+    void* tab = (RULE == DLM_RULE_DECENTLAM) ? (void*)(gs + (size_t)a.n * C) : (void*)gs;
+    const Tables t = stage_tables(a, tab, tables_in_smem != 0);
+    const GT* g = reinterpret_cast<const GT*>(a.g);
+    const int items = a.n << cv_shift;
+    const int cv_mask = (1 << cv_shift) - 1;
+
+    for (long long tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+        const long long c_base = tile * C;
+        __syncthreads();  // previous tile fully consumed (and tables staged on the first pass)
+        for (int e = threadIdx.x; e < items; e += kThreads) {
+            const int i = e >> cv_shift, off = (e & cv_mask) * VEC;
+            const long long c = c_base + off;
+            if (c < a.d) {
+                const Pack<VEC> xi = ld_f32<VEC>(a.x + (size_t)i * a.ld + c);
+                const Pack<VEC> gi = ld_g<VEC>(g + (size_t)i * a.ldg + c);
+                if (RULE == DLM_RULE_DECENTLAM) {
+                    st_f32<VEC>(xs + (size_t)i * C + off, xi);
+                    st_f32<VEC>(gs + (size_t)i * C + off, gi);
+                } else {
+                    const Pack<VEC> mi = ld_f32<VEC>(a.m + (size_t)i * a.ld + c);
+                    Pack<VEC> mn, y;
+#pragma unroll
+                    for (int u = 0; u < VEC; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], y.v[u]);
+                    st_f32<VEC>(a.m + (size_t)i * a.ld + c, mn);
+                    st_f32<VEC>(xs + (size_t)i * C + off, y);
+                }
+            }
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < items; e += kThreads) {
+            const int i = e >> cv_shift, off = (e & cv_mask) * VEC;
+            const long long c = c_base + off;
+            if (c < a.d) {
+                Pack<VEC> xn;
+                if (RULE == DLM_RULE_DECENTLAM) {
+                    const Pack<VEC> mi = ld_f32<VEC>(a.m + (size_t)i * a.ld + c);
+                    Pack<VEC> mn;
+                    decentlam_item<VEC, float>(t, i, off, C, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
+                    st_f32<VEC>(a.m + (size_t)i * a.ld + c, mn);
+                } else {
+                    dmsgd_item<VEC>(t, i, off, C, xs, xn);
+                }
+                st_f32<VEC>(a.x + (size_t)i * a.ld + c, xn);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-bulk-copy pipeline kernel.
+// Shared memory per stage: x tile [n][C] fp32 | m tile [n][C] fp32 | g tile [n][C] GT, each
+// rounded up to 128 bytes; then `stages` mbarriers; then the tables.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 32) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+
+struct TmaGeom {
+    int C;           // tile columns (power of two, multiple of 4... 8 for bf16 g)
+    int cv_shift;    // log2(C / 4)
+    int stages;
+    uint32_t x_bytes, g_bytes, stage_bytes;  // per-stage tile sizes (128-byte multiples)
+    uint32_t tx_bytes;                       // bytes one stage's three copies deliver
+    int tables_in_smem;
+    long long num_tiles;
+};
+
+template <int RULE, typename GT>
+__global__ void __launch_bounds__(kThreads) step_tma_kernel(const __grid_constant__ CUtensorMap tm_x,
+                                                             const __grid_constant__ CUtensorMap tm_m,
+                                                             const __grid_constant__ CUtensorMap tm_g,
+                                                             dlm_step_args a, TmaGeom geo) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    // 128-byte aligned base for the bulk-copy destinations
+    unsigned char* base = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
+    unsigned char* after_stages = base + (size_t)geo.stages * geo.stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(after_stages);
+    void* tab = after_stages + kMaxStages * sizeof(uint64_t);
+    const Tables t = stage_tables(a, tab, geo.tables_in_smem != 0);
+
+    const long long first = blockIdx.x;
+    const long long my_tiles = first < geo.num_tiles ? (geo.num_tiles - first + gridDim.x - 1) / gridDim.x : 0;
+    const int C = geo.C;
+    const int items = a.n << geo.cv_shift;
+    const int cv_mask = (1 << geo.cv_shift) - 1;
+
+    auto issue = [&](int s, long long tile) {
+        const uint32_t bar = smem_u32(&bars[s]);
+        const uint32_t dst = smem_u32(base + (size_t)s * geo.stage_bytes);
+        const int c0 = (int)(tile * C);
+        mbar_expect_tx(bar, geo.tx_bytes);
+        tma_load_2d(dst, &tm_x, c0, 0, bar);
+        tma_load_2d(dst + geo.x_bytes, &tm_m, c0, 0, bar);
+        tma_load_2d(dst + 2 * geo.x_bytes, &tm_g, c0, 0, bar);
+    };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < geo.stages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        for (int s = 0; s < geo.stages && s < my_tiles; ++s) issue(s, first + (long long)s * gridDim.x);
+
+    for (long long it = 0; it < my_tiles; ++it) {
+        const int s = (int)(it % geo.stages);
+        const uint32_t parity = (uint32_t)((it / geo.stages) & 1);
+        const bool arrived = mbar_wait(smem_u32(&bars[s]), parity);
+        if (!__syncthreads_and(arrived)) {  // uniform decision: give up together
+            if (threadIdx.x == 0) {
+                atomicExch(&g_kernel_error, 1);
+                // let copies already issued into the other stages land (bounded) before the CTA's
+                // shared memory is released
+                for (long long j = it + 1; j < my_tiles && j < it + geo.stages; ++j)
+                    mbar_wait(smem_u32(&bars[j % geo.stages]), (uint32_t)((j / geo.stages) & 1));
+            }
+            __syncthreads();
+            return;
+        }
+        unsigned char* st = base + (size_t)s * geo.stage_bytes;
+        float* xs = reinterpret_cast<float*>(st);
+        const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes);
+        const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes);
+        const long long c_base = (first + it * gridDim.x) * C;
+
+        if (RULE == DLM_RULE_DMSGD) {
+            for (int e = threadIdx.x; e < items; e += kThreads) {
+                const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+                const long long c = c_base + off;
+                if (c < a.d) {
+                    const Pack<4> xi = ld_f32<4>(xs + (size_t)i * C + off);
+                    const Pack<4> mi = ld_f32<4>(ms + (size_t)i * C + off);
+                    const Pack<4> gi = ld_g<4>(gs + (size_t)i * C + off);
+                    Pack<4> mn, y;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], y.v[u]);
+                    st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                    st_f32<4>(xs + (size_t)i * C + off, y);
+                }
+            }
+            __syncthreads();
+        }
+        for (int e = threadIdx.x; e < items; e += kThreads) {
+            const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+            const long long c = c_base + off;
+            if (c < a.d) {
+                Pack<4> xn;
+                if (RULE == DLM_RULE_DECENTLAM) {
+                    const Pack<4> mi = ld_f32<4>(ms + (size_t)i * C + off);
+                    Pack<4> mn;
+                    decentlam_item<4, GT>(t, i, off, C, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
+                    st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                } else {
+                    dmsgd_item<4>(t, i, off, C, xs, xn);
+                }
+                st_f32<4>(a.x + (size_t)i * a.ld + c, xn);
+            }
+        }
+        // order this thread's shared-memory accesses before the bulk copy that refills the stage
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (threadIdx.x == 0 && it + geo.stages < my_tiles) issue(s, first + (it + geo.stages) * gridDim.x);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+struct DeviceInfo {
+    int sms = 0;
+    int smem_optin = 0;
+    bool ok = false;
+};
+
+const DeviceInfo& device_info() {
+    static DeviceInfo info[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        static DeviceInfo bad;
+        return bad;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!info[dev].ok) {
+        cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&info[dev].smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        info[dev].ok = info[dev].sms > 0;
+    }
+    return info[dev];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+// 2-D map over a row-major [n, d] array with row stride ld elements; box = [n rows, C columns].
+bool make_map(CUtensorMap* map, const void* ptr, bool bf16, int n, int64_t d, int64_t ld, int C) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t esz = bf16 ? 2 : 4;
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+    cuuint32_t box[2] = {(cuuint32_t)C, (cuuint32_t)n};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                    const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int ilog2(int v) {
+    int l = 0;
+    while ((1 << (l + 1)) <= v) ++l;
+    return l;
+}
+
+size_t table_bytes(const dlm_step_args& a) { return (size_t)(a.n + 1) * 4 + (size_t)a.nnz * 8; }
+
+int g_tune_path = 0;    // 0 auto, 1 force tile kernel, 2 force pipeline kernel (error if ineligible)
+int g_tune_cols = 0;    // tile columns, 0 = auto
+int g_tune_stages = 0;  // pipeline stages, 0 = auto
+int g_tune_ctas = 0;    // CTAs per SM, 0 = auto
+
+template <int RULE, typename GT, int VEC>
+int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return DLM_ERR_CUDA;
+    const int arrays = (RULE == DLM_RULE_DECENTLAM) ? 2 : 1;
+    // widest power-of-two tile with about 64 KB of staged data (at least VEC columns)
+    int C = 1 << ilog2(std::max(1, (int)(65536 / ((size_t)a.n * 4 * arrays))));
+    C = std::max(C, VEC);
+    C = std::min(C, 2048);
+    if (g_tune_cols >= VEC && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
+    while ((long long)C / 2 >= a.d && C / 2 >= VEC) C /= 2;
+    // small problems: prefer enough tiles to occupy every SM over wide tiles
+    while (C / 2 >= 32 * VEC && (a.d + C - 1) / C < dev.sms) C /= 2;
+    size_t tile_bytes = (size_t)a.n * C * 4 * arrays;
+    if (tile_bytes + 16 > (size_t)dev.smem_optin) return DLM_ERR_UNSUPPORTED;
+    int tables_in_smem = tile_bytes + table_bytes(a) + 16 <= (size_t)std::min(dev.smem_optin, 112 * 1024);
+    size_t smem = tile_bytes + (tables_in_smem ? table_bytes(a) : 0) + 16;
+    long long num_tiles = (a.d + C - 1) / C;
+    auto kern = step_tile_kernel<RULE, GT, VEC>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    int per_sm = std::max(1, std::min(8, (int)((size_t)dev.smem_optin / (smem + 1024))));
+    long long grid = std::min<long long>(num_tiles, (long long)dev.sms * per_sm);
+    kern<<<(unsigned)grid, kThreads, smem, stream>>>(a, C, ilog2(C / VEC), tables_in_smem, num_tiles);
+    dlm_count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
+
+// Returns DLM_OK if launched, DLM_ERR_UNSUPPORTED if this shape cannot use the pipeline kernel.
+template <int RULE, typename GT>
+int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return DLM_ERR_CUDA;
+    const bool bf16 = sizeof(GT) == 2;
+    const int min_c = bf16 ? 8 : 4;  // 16-byte inner box extent
+    if (a.n > 256 || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
+    const size_t tab = table_bytes(a);
+    const size_t fixed = 128 + kMaxStages * 8 + 16;
+    const size_t budget = (size_t)dev.smem_optin;
+    int ctas = g_tune_ctas > 0 ? g_tune_ctas : 2;
+    auto stage_bytes_for = [&](int C, uint32_t& xb, uint32_t& gb) {
+        xb = (uint32_t)(((size_t)a.n * C * 4 + 127) & ~(size_t)127);
+        gb = (uint32_t)(((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127);
+        return (size_t)2 * xb + gb;
+    };
+    // tile width: aim at ~16 KB per staged array, at most 256 columns (box limit), at least 16 bytes
+    int C = 1 << ilog2(std::max(1, (int)(16384 / ((size_t)a.n * 4))));
+    C = std::max(min_c, std::min(256, C));
+    if (g_tune_cols >= min_c && g_tune_cols <= 256 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
+    uint32_t xb, gb;
+    size_t sb = stage_bytes_for(C, xb, gb);
+    int tables_in_smem = tab <= 32 * 1024;
+    size_t tabs = tables_in_smem ? tab : 0;
+    int stages = 0;
+    for (; ctas >= 1; --ctas) {
+        size_t per_cta = budget / ctas - (ctas > 1 ? 1024 : 0);
+        if (per_cta < fixed + tabs + sb) continue;
+        stages = (int)std::min<size_t>(kMaxStages, (per_cta - fixed - tabs) / sb);
+        if (stages >= 2 || ctas == 1) break;
+    }
+    if (stages < 2) {  // narrow the tile until two stages fit in one CTA
+        ctas = 1;
+        while (C > min_c) {
+            C /= 2;
+            sb = stage_bytes_for(C, xb, gb);
+            if (budget >= fixed + tabs + 2 * sb) break;
+        }
+        if (budget < fixed + tabs + 2 * sb) return DLM_ERR_UNSUPPORTED;
+        stages = (int)std::min<size_t>(kMaxStages, (budget - fixed - tabs) / sb);
+    }
+    if (g_tune_stages >= 1 && g_tune_stages <= stages) stages = g_tune_stages;
+
+    CUtensorMap tm_x, tm_m, tm_g;
+    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, C) || !make_map(&tm_m, a.m, false, a.n, a.d, a.ld, C) ||
+        !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, C))
+        return DLM_ERR_UNSUPPORTED;
+
+    TmaGeom geo;
+    geo.C = C;
+    geo.cv_shift = ilog2(C / 4);
+    geo.stages = stages;
+    geo.x_bytes = xb;
+    geo.g_bytes = gb;
+    geo.stage_bytes = (uint32_t)sb;
+    geo.tx_bytes = (uint32_t)((size_t)a.n * C * (8 + sizeof(GT)));
+    geo.tables_in_smem = tables_in_smem;
+    geo.num_tiles = (a.d + C - 1) / C;
+    size_t smem = fixed + tabs + (size_t)stages * sb;
+    auto kern = step_tma_kernel<RULE, GT>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    long long grid = std::min<long long>(geo.num_tiles, (long long)dev.sms * ctas);
+    kern<<<(unsigned)grid, kThreads, smem, stream>>>(tm_x, tm_m, tm_g, a, geo);
+    dlm_count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
+
+template <int RULE, typename GT>
+int launch_rule(const dlm_step_args& a, cudaStream_t stream) {
+    const bool bf16 = sizeof(GT) == 2;
+    const uintptr_t px = (uintptr_t)a.x, pm = (uintptr_t)a.m, pg = (uintptr_t)a.g;
+    // 128-bit path: 16-byte aligned bases and rows (bf16 g: 16-byte rows for the bulk copy, 8-byte otherwise)
+    const bool vec_ok = (px % 16 == 0) && (pm % 16 == 0) && (a.ld % 4 == 0) &&
+                        (pg % (bf16 ? 8 : 16) == 0) && (a.ldg % 4 == 0);
+    const bool tma_ok = vec_ok && (pg % 16 == 0) && (a.ldg % (bf16 ? 8 : 4) == 0);
+    if (!vec_ok) {
+        if (g_tune_path == 2) return DLM_ERR_UNSUPPORTED;
+        return launch_tile<RULE, GT, 1>(a, stream);
+    }
+    const int64_t d4 = a.d & ~(int64_t)3;
+    int rc = DLM_OK;
+    if (d4 > 0) {
+        dlm_step_args b = a;
+        b.d = d4;
+        rc = DLM_ERR_UNSUPPORTED;
+        // tiny problems are latency-bound: the plain kernel starts faster than the pipeline
+        const bool want_tma = tma_ok && g_tune_path != 1 && (g_tune_path == 2 || (int64_t)a.n * d4 >= (1 << 20));
+        if (want_tma) rc = launch_tma<RULE, GT>(b, stream);
+        if (rc == DLM_ERR_UNSUPPORTED) {
+            if (g_tune_path == 2) return rc;
+            rc = launch_tile<RULE, GT, 4>(b, stream);
+        }
+        if (rc != DLM_OK) return rc;
+    }
+    if (d4 < a.d) {  // last d mod 4 columns: same arithmetic, scalar accesses
+        dlm_step_args b = a;
+        b.d = a.d - d4;
+        b.x = a.x + d4;
+        b.m = a.m + d4;
+        b.g = (const unsigned char*)a.g + d4 * sizeof(GT);
+        rc = launch_tile<RULE, GT, 1>(b, stream);
+    }
+    return rc;
+}
+
+}  // namespace
+
+int dlm_launch_step(int rule, const dlm_step_args& a, void* stream) {
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (rule == DLM_RULE_DECENTLAM)
+        return a.g_dtype == DLM_G_BF16 ? launch_rule<DLM_RULE_DECENTLAM, __nv_bfloat16>(a, s)
+                                       : launch_rule<DLM_RULE_DECENTLAM, float>(a, s);
+    return a.g_dtype == DLM_G_BF16 ? launch_rule<DLM_RULE_DMSGD, __nv_bfloat16>(a, s)
+                                   : launch_rule<DLM_RULE_DMSGD, float>(a, s);
+}
+
+extern "C" {
+
+DLM_API int dlm_set_tuning(int knob, int value) {
+    switch (knob) {
+    case 0: g_tune_path = value; return DLM_OK;
+    case 1: g_tune_cols = value; return DLM_OK;
+    case 2: g_tune_stages = value; return DLM_OK;
+    case 3: g_tune_ctas = value; return DLM_OK;
+    default: return DLM_ERR_KIND;
+    }
+}
+
+DLM_API int dlm_kernel_error(int* flag) {
+    if (!flag) return DLM_ERR_NULL;
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_kernel_error, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
+    if (v != 0) {
+        int zero = 0;
+        if (cudaMemcpyToSymbol(g_kernel_error, &zero, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
+    }
+    *flag = v;
+    return DLM_OK;
+}
+
+}  // extern "C"

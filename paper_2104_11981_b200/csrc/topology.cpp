@@ -1,0 +1,246 @@
+// Host-side topology builder: neighbour lists and weights per time slot, as CSR tables
+// (Sec. 3 "Network topology and weights": w_ij > 0 iff j is in N_i, and N_i contains i;
+// Assumption A.3: unit row sums; App. G: the graphs used in the experiments).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <new>
+
+#include "dlm_internal.h"
+
+namespace {
+
+struct Edge {
+    int32_t j;
+    int q;  // weight = 1/q
+};
+
+int hops_of(int n) {  // floor(log2(n-1)) + 1, n >= 2
+    int L = 0;
+    while ((int64_t(1) << L) <= n - 1) ++L;
+    return L;
+}
+
+// Finish one row: off-diagonal weights 1/q rounded to fp32, diagonal = fl32(1 - sum 1/q) with
+// the sum taken in double over ascending j; emit columns in ascending order with the self entry.
+void emit_row(int i, std::vector<Edge> nb, dlm_slot& s) {
+    std::sort(nb.begin(), nb.end(), [](const Edge& a, const Edge& b) { return a.j < b.j; });
+    double off = 0.0;
+    for (const Edge& e : nb) off += 1.0 / (double)e.q;
+    float diag = (float)(1.0 - off);
+    bool self_done = false;
+    for (const Edge& e : nb) {
+        if (!self_done && e.j > i) {
+            s.col.push_back(i);
+            s.val.push_back(diag);
+            self_done = true;
+        }
+        s.col.push_back(e.j);
+        s.val.push_back((float)(1.0 / (double)e.q));
+    }
+    if (!self_done) {
+        s.col.push_back(i);
+        s.val.push_back(diag);
+    }
+    s.rowptr.push_back((int32_t)s.col.size());
+    s.max_degree = std::max(s.max_degree, (int)nb.size() + 1);
+}
+
+// Merge duplicate neighbours (several hops landing on the same node), dropping i itself.
+std::vector<Edge> unique_neighbours(int i, const std::vector<int32_t>& js, int q) {
+    std::vector<int32_t> u(js);
+    std::sort(u.begin(), u.end());
+    u.erase(std::unique(u.begin(), u.end()), u.end());
+    std::vector<Edge> nb;
+    for (int32_t j : u)
+        if (j != i) nb.push_back({j, q});
+    return nb;
+}
+
+int upload(dlm_slot& s) {
+    size_t nr = s.rowptr.size() * sizeof(int32_t), nc = s.col.size() * sizeof(int32_t),
+           nv = s.val.size() * sizeof(float);
+    if (cudaMalloc((void**)&s.d_rowptr, nr) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMalloc((void**)&s.d_col, nc) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMalloc((void**)&s.d_val, nv) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_rowptr, s.rowptr.data(), nr, cudaMemcpyHostToDevice) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_col, s.col.data(), nc, cudaMemcpyHostToDevice) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_val, s.val.data(), nv, cudaMemcpyHostToDevice) != cudaSuccess) return DLM_ERR_CUDA;
+    return DLM_OK;
+}
+
+// Validate a caller-supplied sparsity pattern: monotone rowptr, in-range ascending unique columns.
+bool pattern_ok(int n, const int32_t* rowptr, const int32_t* col) {
+    if (rowptr[0] != 0) return false;
+    for (int i = 0; i < n; ++i) {
+        if (rowptr[i + 1] < rowptr[i]) return false;
+        for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+            if (col[p] < 0 || col[p] >= n) return false;
+            if (p > rowptr[i] && col[p] <= col[p - 1]) return false;
+        }
+    }
+    return true;
+}
+
+bool has_entry(const int32_t* rowptr, const int32_t* col, int i, int j) {
+    return std::binary_search(col + rowptr[i], col + rowptr[i + 1], (int32_t)j);
+}
+
+}  // namespace
+
+extern "C" {
+
+int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
+                   dlm_topology** out) {
+    if (!out) return DLM_ERR_NULL;
+    *out = nullptr;
+    if (kind < DLM_TOPO_RING || kind > DLM_TOPO_CSR_WEIGHTS) return DLM_ERR_KIND;
+    if (n < 1) return DLM_ERR_SHAPE;
+    if (n > DLM_MAX_NODES) return DLM_ERR_UNSUPPORTED;
+    if (kind == DLM_TOPO_RING && n < 3) return DLM_ERR_SHAPE;
+    if ((kind == DLM_TOPO_STATIC_EXP || kind == DLM_TOPO_ONE_PEER_EXP) && n < 2) return DLM_ERR_SHAPE;
+    if (kind == DLM_TOPO_CSR_MH && (!rowptr || (!col && rowptr[n] > 0))) return DLM_ERR_NULL;
+    if (kind == DLM_TOPO_CSR_WEIGHTS && (!rowptr || !col || !val)) return DLM_ERR_NULL;
+
+    dlm_topology* t = new (std::nothrow) dlm_topology;
+    if (!t) return DLM_ERR_CUDA;
+    t->n = n;
+    t->kind = kind;
+    int period = (kind == DLM_TOPO_ONE_PEER_EXP) ? hops_of(n) : 1;
+    t->slots.resize(period);
+    int rc = DLM_OK;
+
+    for (int slot = 0; slot < period && rc == DLM_OK; ++slot) {
+        dlm_slot& s = t->slots[slot];
+        s.rowptr.push_back(0);
+        switch (kind) {
+        case DLM_TOPO_RING:
+            for (int i = 0; i < n; ++i)
+                emit_row(i, unique_neighbours(i, {(int32_t)((i + 1) % n), (int32_t)((i + n - 1) % n)}, 3), s);
+            break;
+        case DLM_TOPO_STATIC_EXP: {
+            int L = hops_of(n);
+            for (int i = 0; i < n; ++i) {
+                std::vector<int32_t> js;
+                for (int h = 0; h < L; ++h) js.push_back((int32_t)(((int64_t)i + (int64_t(1) << h)) % n));
+                emit_row(i, unique_neighbours(i, js, L + 1), s);
+            }
+            break;
+        }
+        case DLM_TOPO_ONE_PEER_EXP:
+            for (int i = 0; i < n; ++i)
+                emit_row(i, unique_neighbours(i, {(int32_t)(((int64_t)i + (int64_t(1) << slot)) % n)}, 2), s);
+            break;
+        case DLM_TOPO_COMPLETE:
+            for (int i = 0; i < n; ++i) {
+                std::vector<Edge> nb;
+                for (int j = 0; j < n; ++j)
+                    if (j != i) nb.push_back({(int32_t)j, n});
+                emit_row(i, nb, s);
+            }
+            break;
+        case DLM_TOPO_CSR_MH: {
+            if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
+            for (int i = 0; i < n && rc == DLM_OK; ++i)
+                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p)
+                    if (col[p] == i || !has_entry(rowptr, col, col[p], i)) { rc = DLM_ERR_TOPOLOGY; break; }
+            if (rc != DLM_OK) break;
+            for (int i = 0; i < n; ++i) {
+                int deg_i = rowptr[i + 1] - rowptr[i];
+                std::vector<Edge> nb;
+                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                    int j = col[p], deg_j = rowptr[j + 1] - rowptr[j];
+                    nb.push_back({(int32_t)j, 1 + std::max(deg_i, deg_j)});
+                }
+                emit_row(i, nb, s);
+            }
+            break;
+        }
+        case DLM_TOPO_CSR_WEIGHTS: {
+            if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
+            std::vector<double> colsum(n, 0.0);
+            for (int i = 0; i < n && rc == DLM_OK; ++i) {
+                double rowsum = 0.0;
+                if (!has_entry(rowptr, col, i, i)) { rc = DLM_ERR_TOPOLOGY; break; }
+                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                    if (!(val[p] > 0.0f) || !std::isfinite(val[p])) { rc = DLM_ERR_TOPOLOGY; break; }
+                    rowsum += (double)val[p];
+                    colsum[col[p]] += (double)val[p];
+                }
+                if (rc == DLM_OK && std::fabs(rowsum - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
+            }
+            for (int j = 0; j < n && rc == DLM_OK; ++j)
+                if (std::fabs(colsum[j] - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
+            if (rc != DLM_OK) break;
+            s.rowptr.assign(rowptr, rowptr + n + 1);
+            s.col.assign(col, col + rowptr[n]);
+            s.val.assign(val, val + rowptr[n]);
+            for (int i = 0; i < n; ++i) s.max_degree = std::max(s.max_degree, rowptr[i + 1] - rowptr[i]);
+            break;
+        }
+        }
+    }
+    // Without a CUDA device the handle stays host-only (tables can be inspected, steps fail).
+    int ndev = 0;
+    bool have_device = rc == DLM_OK && cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0;
+    if (rc == DLM_OK && !have_device) cudaGetLastError();
+    if (have_device && cudaGetDevice(&t->device) != cudaSuccess) rc = DLM_ERR_CUDA;
+    for (int slot = 0; have_device && slot < period && rc == DLM_OK; ++slot) rc = upload(t->slots[slot]);
+    if (rc != DLM_OK) {
+        cudaGetLastError();  // clear the error left by a failed runtime call
+        topology_destroy(t);
+        return rc;
+    }
+    *out = t;
+    return DLM_OK;
+}
+
+int topology_period(const dlm_topology* topo, int* period) {
+    if (!topo || !period) return DLM_ERR_NULL;
+    *period = (int)topo->slots.size();
+    return DLM_OK;
+}
+
+int topology_nodes(const dlm_topology* topo, int* n) {
+    if (!topo || !n) return DLM_ERR_NULL;
+    *n = topo->n;
+    return DLM_OK;
+}
+
+int topology_tables_host(const dlm_topology* topo, int slot, const int32_t** rowptr, const int32_t** col,
+                         const float** val, int64_t* nnz) {
+    if (!topo) return DLM_ERR_NULL;
+    if (slot < 0 || slot >= (int)topo->slots.size()) return DLM_ERR_SHAPE;
+    const dlm_slot& s = topo->slots[slot];
+    if (rowptr) *rowptr = s.rowptr.data();
+    if (col) *col = s.col.data();
+    if (val) *val = s.val.data();
+    if (nnz) *nnz = (int64_t)s.col.size();
+    return DLM_OK;
+}
+
+int topology_tables_device(const dlm_topology* topo, int slot, const int32_t** rowptr, const int32_t** col,
+                           const float** val, int64_t* nnz) {
+    if (!topo) return DLM_ERR_NULL;
+    if (slot < 0 || slot >= (int)topo->slots.size()) return DLM_ERR_SHAPE;
+    const dlm_slot& s = topo->slots[slot];
+    if (rowptr) *rowptr = s.d_rowptr;
+    if (col) *col = s.d_col;
+    if (val) *val = s.d_val;
+    if (nnz) *nnz = (int64_t)s.col.size();
+    return DLM_OK;
+}
+
+int topology_destroy(dlm_topology* topo) {
+    if (!topo) return DLM_OK;
+    for (dlm_slot& s : topo->slots) {
+        if (s.d_rowptr) cudaFree(s.d_rowptr);
+        if (s.d_col) cudaFree(s.d_col);
+        if (s.d_val) cudaFree(s.d_val);
+    }
+    delete topo;
+    return DLM_OK;
+}
+
+}  // extern "C"

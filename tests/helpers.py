@@ -1,0 +1,63 @@
+"""Shared test plumbing: maps a workload to both sides' topologies, moves data, measures errors.
+No update-rule arithmetic lives here."""
+import os
+
+import numpy as np
+
+import oracle
+from paper_2104_11981_b200 import inputs
+
+ORACLE_KIND = {"ring": oracle.RING, "static_exp": oracle.STATIC_EXP, "one_peer_exp": oracle.ONE_PEER_EXP,
+               "complete": oracle.COMPLETE, "er_mh": oracle.ADJ_MH}
+THREADS = max(1, os.cpu_count() or 1)
+
+
+def build_both(topology, n, graph_seed=None, er_p=0.05):
+    """Returns (library Topology, [dense oracle W per slot])."""
+    from paper_2104_11981_b200 import binding as B
+    lib_kind = {"ring": B.RING, "static_exp": B.STATIC_EXP, "one_peer_exp": B.ONE_PEER_EXP,
+                "complete": B.COMPLETE, "er_mh": B.CSR_MH}[topology]
+    adj = None
+    if topology == "er_mh":
+        adj, _ = inputs.er_adjacency(n, er_p, graph_seed)
+        rowptr, col = inputs.adjacency_to_lists(adj)
+        topo = B.topology_build(lib_kind, n, rowptr, col)
+    else:
+        topo = B.topology_build(lib_kind, n)
+    ok = ORACLE_KIND[topology]
+    Ws = [oracle.topology_dense(ok, n, s, adj) for s in range(oracle.topology_period(ok, n))]
+    assert topo.period == len(Ws)
+    return topo, Ws
+
+
+def rel_l2(a, o):
+    """||a - o||_2 / ||o||_2 over the whole tensor; exact zero required when the oracle is zero."""
+    a = np.asarray(a, dtype=np.float64); o = np.asarray(o, dtype=np.float64)
+    den = np.linalg.norm(o)
+    if den == 0.0:
+        return 0.0 if np.linalg.norm(a) == 0.0 else np.inf
+    return float(np.linalg.norm(a - o) / den)
+
+
+def to64(t):
+    """torch tensor (fp32 or bf16, any device) -> float64 numpy (exact)."""
+    import torch
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def oracle_rule(rule, W, x, m, g, beta, gamma, threads=THREADS):
+    if rule == "decentlam":
+        return oracle.decentlam_step(W, x, m, g, beta, gamma, threads)
+    if rule == "dmsgd":
+        return oracle.dmsgd_step(W, x, m, g, beta, gamma, threads)
+    return oracle.pmsgd_step(x, m, g, beta, gamma, threads)
+
+
+def lib_rule(rule, topo, k, x, m, g, beta, gamma):
+    from paper_2104_11981_b200 import binding as B
+    if rule == "decentlam":
+        B.decentlam_step(topo, k, x, m, g, beta, gamma)
+    elif rule == "dmsgd":
+        B.dmsgd_step(topo, k, x, m, g, beta, gamma)
+    else:
+        B.pmsgd_step(x, m, g, beta, gamma)

@@ -1,0 +1,124 @@
+"""GPU parity for the least-squares gradient kernel and the convex end-to-end workload (cfg4)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import THREADS, build_both, lib_rule, oracle_rule, rel_l2, to64
+from paper_2104_11981_b200 import inputs
+from paper_2104_11981_b200.inputs import WORKLOADS, seed_for
+
+pytestmark = pytest.mark.gpu
+# fp32 dot products of length q and p with warp-tree partial sums against a double oracle:
+# error ~ eps * sqrt(length) of the accumulated magnitude; 2e-6 relative L2 leaves a 4x margin.
+TOL_LSQ = 2e-6
+
+
+def _lsq_gpu(A, b, x, scale):
+    from paper_2104_11981_b200 import binding as B
+    n, p, q = A.shape
+    ws = torch.empty(B.lsq_grad_workspace_bytes(n, p, q), dtype=torch.uint8, device=A.device)
+    g = torch.full((n, q), float("nan"), device=A.device)
+    B.lsq_grad(A, b, x, g, scale, ws)
+    return g
+
+
+@pytest.mark.parametrize("n,p,q", [(1, 1, 1), (3, 50, 30), (8, 50, 30), (2, 7, 128), (4, 100, 256), (5, 333, 384),
+                                    (3, 64, 1024), (2, 40, 1000), (2, 9, 4100), (32, 4096, 1024)])
+def test_lsq_grad_matches_oracle(n, p, q):
+    dev = torch.device("cuda:0")
+    A, b, _ = inputs.lsq_problem_torch(n, p, q, 100 + n + p + q, dev)
+    x = inputs.normal_torch((n, q), 1.0, 7 + q, dev)
+    scale = 1.0 / p
+    g = _lsq_gpu(A, b, x, scale)
+    go = oracle.lsq_grad(A.cpu().numpy(), b.cpu().numpy(), to64(x), np.float32(scale), THREADS)
+    assert torch.isfinite(g).all()
+    assert rel_l2(to64(g), go) <= TOL_LSQ
+    g2 = _lsq_gpu(A, b, x, scale)
+    assert torch.equal(g, g2)                     # fixed summation order: bitwise repeatable
+
+
+def test_lsq_grad_near_a_minimiser():
+    """At x_i = argmin f_i the gradient is pure cancellation: the residual A x - b is formed from
+    terms of size |A||x| + |b|, so the error is judged against |A|^T (|A||x| + |b|) * scale."""
+    dev = torch.device("cuda:0")
+    n, p, q = 4, 512, 128
+    A, b, _ = inputs.lsq_problem_torch(n, p, q, 5, dev)
+    xs = torch.linalg.lstsq(A.double(), b.double().unsqueeze(-1)).solution.squeeze(-1).float()
+    g = _lsq_gpu(A, b, xs, 1.0 / p)
+    go = oracle.lsq_grad(A.cpu().numpy(), b.cpu().numpy(), to64(xs), np.float32(1.0 / p))
+    Aa = A.abs().double()
+    inner = torch.bmm(Aa, xs.abs().double().unsqueeze(-1)).squeeze(-1) + b.abs().double()      # [n, p]
+    terms = torch.bmm(Aa.transpose(1, 2), inner.unsqueeze(-1)).squeeze(-1) / p                  # [n, q]
+    assert np.max(np.abs(to64(g) - go) / terms.cpu().numpy()) < 2e-7
+
+
+def _cfg4_run(n, p, q, steps, rule, gamma, beta, seed, oracle_steps):
+    """GPU loop lsq_grad -> step for `steps` iterations; the oracle free-runs for the first
+    `oracle_steps`.  Returns (A, b, x_gpu, rel errors at oracle_steps)."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    A, b, _ = inputs.lsq_problem_torch(n, p, q, seed, dev)
+    topo, Ws = build_both("ring", n)
+    ws = torch.empty(B.lsq_grad_workspace_bytes(n, p, q), dtype=torch.uint8, device=dev)
+    x = torch.zeros((n, q), device=dev); m = torch.zeros_like(x); g = torch.empty_like(x)
+    An, bn = A.cpu().numpy(), b.cpu().numpy()
+    xo = np.zeros((n, q)); mo = np.zeros((n, q))
+    scale = 1.0 / p
+    errs = None
+    for k in range(steps):
+        B.lsq_grad(A, b, x, g, scale, ws)
+        if rule == "pmsgd":
+            B.pmsgd_step(x, m, g, beta, gamma)
+        else:
+            lib_rule(rule, topo, k, x, m, g, beta, gamma)
+        if k < oracle_steps:
+            go = oracle.lsq_grad(An, bn, xo, np.float32(scale), THREADS)
+            xo, mo = oracle_rule(rule, Ws[0], xo, mo, go, np.float32(beta), np.float32(gamma))
+            if k == oracle_steps - 1:
+                # m tends to 0 for DecentLaM and PmSGD as the run converges; it is then judged against
+                # the gradient it is built from (the larger operand), not against its own vanishing norm
+                em = np.linalg.norm(to64(m) - mo) / max(np.linalg.norm(mo), np.linalg.norm(go))
+                errs = (rel_l2(to64(x), xo), float(em))
+    torch.cuda.synchronize()
+    assert B.kernel_error() == 0
+    return An, bn, Ws[0], to64(x), errs
+
+
+@pytest.mark.parametrize("rule", ["decentlam", "dmsgd", "pmsgd"])
+def test_cfg4_reduced_size_full_run(rule):
+    """Same recipe at n=8, p=256, q=128: the oracle follows all 2000 iterations."""
+    w = WORKLOADS["cfg4"]
+    _, _, _, _, errs = _cfg4_run(8, 256, 128, w.steps, rule, w.gamma, w.beta, seed_for("cfg4", inputs.P_LSQ), w.steps)
+    assert errs[0] <= 1e-4 and errs[1] <= 1e-4, errs
+
+
+def test_cfg4_full_size():
+    """n=32, A_i [4096, 1024], ring, beta=0.9, gamma=0.01, 2000 steps of DecentLaM and DmSGD.
+    The oracle follows the first 60 iterations element by element; the end state is checked
+    through what App. C fixes: DecentLaM's limit solves (I-W)X = -gamma W grad f(X), DmSGD's
+    solves (1-beta)(I-W)X = -gamma W grad f(X), the averaged gradient vanishes at both, and
+    DecentLaM ends closer to the closed-form optimum than DmSGD."""
+    w = WORKLOADS["cfg4"]
+    seed = seed_for("cfg4", inputs.P_LSQ)
+    out = {}
+    for rule in ("decentlam", "dmsgd"):
+        An, bn, W, x, errs = _cfg4_run(w.n, w.p, w.d, w.steps, rule, w.gamma, w.beta, seed, 60)
+        assert errs[0] <= 1e-4 and errs[1] <= 1e-4, (rule, errs)
+        out[rule] = x
+    xstar = oracle.lsq_optimum(An, bn)
+    off = W.copy(); np.fill_diagonal(off, 0.0)
+    L = np.diag(off.sum(1)) - off
+    Wexact = off + np.diag(1.0 - off.sum(1))
+    gamma, beta = np.float64(np.float32(w.gamma)), np.float64(np.float32(w.beta))
+    for rule, coeff, Wg in (("decentlam", 1.0, W), ("dmsgd", 1.0 - beta, Wexact)):
+        x = out[rule]
+        grad = oracle.lsq_grad(An, bn, x, np.float32(1.0 / w.p), THREADS)
+        lhs, rhs = coeff * (L @ x), -gamma * (Wg @ grad)
+        # fp32 state: the residual is limited by the rounding of x itself, ~ 2^-24 ||x|| in (I-W)x;
+        # a wrong fixed point (e.g. the other rule's) would leave a residual of order ||rhs||
+        assert np.linalg.norm(lhs - rhs) <= 3 * 2.0 ** -24 * np.linalg.norm(x), rule
+        assert np.linalg.norm(lhs - rhs) <= 1e-3 * np.linalg.norm(rhs), rule
+        assert np.linalg.norm(grad.mean(0)) <= 2e-4 * np.linalg.norm(grad) / np.sqrt(w.n)
+    el, em = oracle.relative_error(out["decentlam"], xstar), oracle.relative_error(out["dmsgd"], xstar)
+    assert el < em and em / el <= 1.0 / (1.0 - beta) ** 2 * 1.01
