@@ -33,10 +33,12 @@ MAX_STEPS_PER_CHUNK = 256   # state is re-initialised (untimed) between chunks: 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--columns", type=int, default=0,
+                    help="override d (columns per node): a smaller case of the same kernel, for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the DmSGD / PmSGD side timings")
@@ -229,7 +231,7 @@ def run_ours(args):
     w = inputs.WORKLOADS[args.workload]
     if w.p:
         raise SystemExit("bench.py times the step workloads (cfg1, cfg2, cfg3, cfg5)")
-    n, d = w.n, w.d
+    n, d = w.n, (args.columns or w.d)
     gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
 
     if w.topology == "er_mh":
@@ -320,7 +322,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
+            "config": {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else ""), "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
                        "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": f"working set {(8 + g.element_size()) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

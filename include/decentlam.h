@@ -192,8 +192,10 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 0  kernel path: 1 = plain-load tile kernel, 2 = bulk-copy pipeline kernel (steps whose
  *           layout cannot use it then return DLM_ERR_UNSUPPORTED)
  *   knob 1  tile width in columns (power of two)
- *   knob 2  pipeline stages
- *   knob 3  CTAs per SM the pipeline kernel sizes its shared memory for
+ *   knob 2  pipeline stages per CTA
+ *   knob 3  CTAs per SM of the persistent grid (used with knob 4 < 0)
+ *   knob 4  tiles per CTA: t > 0 launches ceil(tiles / t) CTAs; t < 0 a persistent grid
+ *   knob 5  neighbour tables: 1 = staged in shared memory, 2 = read from global memory
  * Results do not depend on the knobs (all paths round identically).  DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);

@@ -115,8 +115,11 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
     g = inputs.normal_torch((n, d), 1e-3, 3, dev, dtype=gt)
     outs = []
     try:
-        for path, cols, stages in ((1, 0, 0), (2, 0, 0), (2, 64, 2), (2, 256, 3), (1, 128, 0)):
+        # (path, tile columns, stages, tiles per CTA, tables)
+        for path, cols, stages, tpc, tab in ((1, 0, 0, 0, 0), (2, 0, 0, 0, 0), (2, 64, 2, -1, 1), (2, 256, 3, -1, 2),
+                                             (2, 512, 2, 4, 0), (2, 32, 1, 3, 2), (1, 128, 0, 0, 0)):
             B.set_tuning(0, path); B.set_tuning(1, cols); B.set_tuning(2, stages)
+            B.set_tuning(4, tpc); B.set_tuning(5, tab)
             x, m = x0.clone(), m0.clone()
             for k in range(3):
                 lib_rule(rule, topo, k, x, m, g, 0.9, 0.1)
@@ -124,7 +127,7 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
             assert B.kernel_error() == 0
             outs.append((x, m))
     finally:
-        for knob in range(4):
+        for knob in range(6):
             B.set_tuning(knob, 0)
     for x, m in outs[1:]:
         assert torch.equal(x, outs[0][0]) and torch.equal(m, outs[0][1])
