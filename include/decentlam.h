@@ -177,6 +177,38 @@ DLM_API int64_t lsq_grad_workspace_bytes(int n, int p, int q); /* negative dlm_s
 DLM_API int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
              float scale, void* workspace, int64_t workspace_bytes, void* cuda_stream);
 
+/*
+ * lsq_grad without any device allocation (the paper has no counterpart: this entry point exists
+ * for the host program's sake, not for the method's).
+ *
+ * Some programs that want this gradient cannot obtain device scratch to hand to lsq_grad: a
+ * plain-C driver that received only its input and output buffers from a framework owning the
+ * rest of the GPU's memory (a cudaMalloc there fails or fights the framework's pool), or a
+ * latency-sensitive loop that must not pay the device-wide synchronisation cudaMalloc and
+ * cudaFree imply.  For them the partial sums live in a fixed array of
+ * DLM_LSQ_STATIC_SCRATCH_BYTES (4 MiB) inside the library's device code.  Each GPU on which the
+ * library runs keeps that array until the process ends.
+ *
+ * Arguments and result are those of lsq_grad (same kernels, same summation order, bitwise the
+ * same g), minus the workspace.  Neither this call nor anything below it calls cudaMalloc,
+ * cudaFree or an allocating library routine.
+ *   - Size limit: n * S * q * 4 bytes must fit the array, S <= 64 being the number of row chunks
+ *     per node the library picks for (n, p) on the current GPU (about 2 * SM count / n).  The cfg4
+ *     problem (n = 32, q = 1024) needs 1.2 MiB.  Larger problems return DLM_ERR_WORKSPACE and
+ *     launch nothing; use lsq_grad with your own workspace instead.
+ *   - First call on a device: looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and caches it; make this first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call left there.  No
+ *     clearing is needed (each call overwrites every partial sum before reading it), but two
+ *     calls whose kernels can overlap on the GPU (different streams, or the same stream from
+ *     two threads without ordering) race on it and give wrong results: order them.
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_UNSUPPORTED (q above
+ *         8192), DLM_ERR_WORKSPACE (problem too large for the built-in scratch), DLM_ERR_CUDA.
+ */
+#define DLM_LSQ_STATIC_SCRATCH_BYTES (4u << 20)
+DLM_API int lsq_grad_static(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
+                            float scale, void* cuda_stream);
+
 /* Kernel launches issued by this library in the calling process so far (all entry points). */
 DLM_API int64_t dlm_launch_count(void);
 

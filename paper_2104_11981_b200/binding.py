@@ -54,6 +54,7 @@ _lib.pmsgd_step.argtypes = [_int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _
 _lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
 _lib.lsq_grad_workspace_bytes.restype = _i64
 _lib.lsq_grad.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp, _i64, _vp]
+_lib.lsq_grad_static.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp]
 _lib.dlm_launch_count.argtypes = []
 _lib.dlm_launch_count.restype = _i64
 _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
@@ -61,7 +62,7 @@ _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_period", "topology_nodes", "topology_tables_host",
            "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "pmsgd_step",
-           "lsq_grad_workspace_bytes", "lsq_grad", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
+           "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
 def _check(rc, where):
@@ -195,6 +196,21 @@ def lsq_grad(A, b, x, g, scale, workspace, stream=None):
     _check(_lib.lsq_grad(n, p, q, _vp(A.data_ptr()), _vp(b.data_ptr()), _vp(x.data_ptr()), _vp(g.data_ptr()),
                          scale, _vp(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
                          _stream_ptr(stream)), "lsq_grad")
+
+
+LSQ_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def lsq_grad_static(A, b, x, g, scale, stream=None):
+    """lsq_grad for callers that cannot allocate device scratch: same arguments minus the
+    workspace, same result.  The partial sums go to a fixed 4 MiB array inside the library, shared
+    by all calls, so calls must not overlap on the GPU; problems whose partial sums do not fit
+    raise DecentlamError(DLM_ERR_WORKSPACE)."""
+    n, p, q = A.shape
+    assert A.is_contiguous() and b.is_contiguous() and x.is_contiguous() and g.is_contiguous()
+    assert b.shape == (n, p) and x.shape == (n, q) and g.shape == (n, q)
+    _check(_lib.lsq_grad_static(n, p, q, _vp(A.data_ptr()), _vp(b.data_ptr()), _vp(x.data_ptr()),
+                                _vp(g.data_ptr()), scale, _stream_ptr(stream)), "lsq_grad_static")
 
 
 def launch_count():

@@ -190,3 +190,64 @@ int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, con
     dlm_count_launch(2);
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------
+// lsq_grad_static: the same computation for callers that cannot allocate device memory.
+// The [n, S, q] partial sums live in a fixed array that is part of the loaded module, so the
+// caller passes inputs and outputs only.  Every device that loads the library holds the
+// array until the process exits.
+// ---------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr size_t kStaticScratchFloats = DLM_LSQ_STATIC_SCRATCH_BYTES / sizeof(float);
+static __device__ __align__(256) float g_lsq_static_scratch[kStaticScratchFloats];
+
+// Device address of the array on the current device.  In host code the array's name is only a
+// handle for the runtime, not something a kernel can dereference, so the address is looked up
+// once per device (with that device current) and cached.
+int static_scratch_address(float** out) {
+    static float* cached[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DLM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_lsq_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return DLM_ERR_CUDA;
+        }
+        cached[dev] = static_cast<float*>(p);
+    }
+    *out = cached[dev];
+    return DLM_OK;
+}
+
+bool ranges_overlap(const void* a, size_t abytes, const void* b, size_t bbytes) {
+    uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bbytes && b0 < a0 + abytes;
+}
+
+}  // namespace
+
+extern "C" DLM_API int lsq_grad_static(int n, int p, int q, const float* A, const float* b, const float* x,
+                                       float* g, float scale, void* cuda_stream) {
+    if (!A || !b || !x || !g) return DLM_ERR_NULL;
+    if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
+    if (q > kGenericMaxQ) return DLM_ERR_UNSUPPORTED;
+    if ((uintptr_t)A % 16 || (uintptr_t)x % 16 || (uintptr_t)g % 16 || (uintptr_t)b % 4) return DLM_ERR_ALIGN;
+    const size_t ab = (size_t)n * p * q * 4, bb = (size_t)n * p * 4, xb = (size_t)n * q * 4;
+    if (ranges_overlap(g, xb, A, ab) || ranges_overlap(g, xb, b, bb) || ranges_overlap(g, xb, x, xb))
+        return DLM_ERR_ALIAS;
+    const int S = dlm_lsq_splits(n, p, q);
+    if (S < 1) return DLM_ERR_CUDA;
+    if ((size_t)n * S * q > kStaticScratchFloats) return DLM_ERR_WORKSPACE;  // beyond the built-in scratch
+    float* scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != DLM_OK) return rc;
+    // Every partial [i, s, :] that the reduction reads is written by the first kernel of this same
+    // call, so nothing left over from an earlier call is ever consumed and nothing needs clearing.
+    return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, scratch, cuda_stream);
+}
