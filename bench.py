@@ -230,7 +230,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     w = inputs.WORKLOADS[args.workload]
     if w.p:
-        raise SystemExit("bench.py times the step workloads (cfg1, cfg2, cfg3, cfg5)")
+        return run_lsq_workload(args, w, B, inputs, torch, dev, rank, world, dist)
     n, d = w.n, (args.columns or w.d)
     gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
 
@@ -331,6 +331,50 @@ def run_ours(args):
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "cpu_baseline": cpu_baseline,
             "other_rules": extra,
         }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_lsq_workload(args, w, B, inputs, torch, dev, rank, world, dist):
+    """cfg4: every iteration is lsq_grad (streams A once) followed by decentlam_step on [n, q]."""
+    n, p, q = w.n, w.p, w.d
+    A, b, _ = inputs.lsq_problem_torch(n, p, q, inputs.seed_for(args.workload, inputs.P_LSQ) + rank, dev)
+    topo = B.topology_build(B.RING, n)
+    ws = torch.empty(B.lsq_grad_workspace_bytes(n, p, q), dtype=torch.uint8, device=dev)
+    x = torch.zeros((n, q), device=dev); m = torch.zeros_like(x); g = torch.empty_like(x)
+    stream = torch.cuda.current_stream()
+    scale = 1.0 / p
+
+    def reset():
+        x.zero_(); m.zero_()
+
+    def iteration(k):
+        B.lsq_grad(A, b, x, g, scale, ws)
+        B.decentlam_step(topo, k, x, m, g, w.beta, w.gamma)
+
+    sampler = ClockSampler(dev.index or 0)
+    if dist is not None:
+        dist.barrier()
+    sampler.start()
+    secs, launches = time_steps(iteration, reset, args.steps, args.warmup, torch, stream, B.launch_count)
+    clocks = sampler.stop()
+    lsq_secs, _ = time_steps(lambda k: B.lsq_grad(A, b, x, g, scale, ws), reset, args.steps, 3, torch, stream)
+    job_secs, job_units = aggregate_over_ranks(dist, secs, n * q * args.steps, dev)
+    peak, peak_kind = measured_peak()
+    lsq_bytes = 4 * (n * p * q + n * p + 2 * n * q)
+    achieved = lsq_bytes * args.steps / lsq_secs / 1e9
+    if rank == 0:
+        line = {"metric": METRIC, "value": job_units / job_secs, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": args.workload, "n": n, "p": p, "q": q, "topology": w.topology, "beta": w.beta,
+                           "gamma": w.gamma, "l2": f"A is {n * p * q * 4 / 2**20:.0f} MiB, larger than the 126 MB L2; no flush"},
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                             "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "lsq_partial_rows_kernel + lsq_reduce_kernel",
+                             "algorithmic_bytes_per_launch": lsq_bytes, "ms_per_lsq_grad": lsq_secs / args.steps * 1e3},
+                "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "cpu_baseline": None}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()

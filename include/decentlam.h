@@ -228,6 +228,8 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 3  CTAs per SM of the persistent grid (used with knob 4 < 0)
  *   knob 4  tiles per CTA: t > 0 launches ceil(tiles / t) CTAs; t < 0 a persistent grid
  *   knob 5  neighbour tables: 1 = staged in shared memory, 2 = read from global memory
+ *   knob 6  threads per CTA of the pipeline kernel (128, 256 or 512)
+ *   knob 7  mixing loop: 1 = warp-cooperative table fetch, 2 = plain per-thread loop
  * Results do not depend on the knobs (all paths round identically).  DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);

@@ -57,6 +57,9 @@ int topo_step(int rule, const dlm_topology* topo, int64_t k, int n, int64_t d, i
     a.rowptr = s.d_rowptr;
     a.col = s.d_col;
     a.val = s.d_val;
+    a.order = s.d_order;
+    a.rows = s.d_rows;
+    a.ent = s.d_ent;
     a.nnz = (int)s.col.size();
     a.max_degree = s.max_degree;
     a.beta = beta;

@@ -9,6 +9,13 @@
 struct dlm_slot {
     std::vector<int32_t> rowptr, col;
     std::vector<float> val;
+    std::vector<int32_t> order;  // rows sorted by decreasing degree (stable): the kernels' processing order
+    int32_t* d_order = nullptr;
+    // packed copies for the warp-cooperative kernels: rows[r] = {i, first entry, length, 0} in
+    // processing order; ent[p] = {col[p], bits of val[p]}
+    std::vector<int32_t> rows, ent;
+    int32_t* d_rows = nullptr;
+    int32_t* d_ent = nullptr;
     int32_t* d_rowptr = nullptr;
     int32_t* d_col = nullptr;
     float* d_val = nullptr;
@@ -35,6 +42,9 @@ struct dlm_step_args {
     const int32_t* rowptr;  // device
     const int32_t* col;     // device
     const float* val;       // device
+    const int32_t* order;   // device, row processing order (a permutation of 0..n-1)
+    const int32_t* rows;    // device, int4 per row in processing order {i, first entry, length, 0}
+    const int32_t* ent;     // device, int2 per entry {col, bits of val}
     int nnz;
     int max_degree;
     float beta, gamma, inv_gamma;

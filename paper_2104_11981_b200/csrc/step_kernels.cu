@@ -24,7 +24,8 @@
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;     // tile kernel block size
+constexpr int kMaxThreads = 512;  // pipeline kernel block size limit
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWaitLimit = 1u << 22;  // polls before a pipeline wait gives up
 
@@ -93,24 +94,28 @@ __device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
     return {{bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(p))}};
 }
 
+
 // Neighbour tables of the current slot, either copied to shared memory or left in global memory.
 struct Tables {
     const int* rowptr;
     const int* col;
     const float* val;
+    const int* order;
 };
 
 __device__ __forceinline__ Tables stage_tables(const dlm_step_args& a, void* smem_tables, bool in_smem) {
-    if (!in_smem) return {a.rowptr, a.col, a.val};
+    if (!in_smem) return {a.rowptr, a.col, a.val, a.order};
     int* s_rowptr = reinterpret_cast<int*>(smem_tables);
-    int* s_col = s_rowptr + (a.n + 1);
+    int* s_order = s_rowptr + (a.n + 1);
+    int* s_col = s_order + a.n;
     float* s_val = reinterpret_cast<float*>(s_col + a.nnz);
     for (int i = threadIdx.x; i <= a.n; i += blockDim.x) s_rowptr[i] = a.rowptr[i];
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s_order[i] = a.order[i];
     for (int i = threadIdx.x; i < a.nnz; i += blockDim.x) {
         s_col[i] = a.col[i];
         s_val[i] = a.val[i];
     }
-    return {s_rowptr, s_col, s_val};
+    return {s_rowptr, s_col, s_val, s_order};
 }
 
 // Mix one item (row i, VEC consecutive columns at tile offset off) of the DecentLaM rule.
@@ -119,19 +124,19 @@ template <int VEC, typename GS>
 __device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, int C, const float* xs,
                                                const GS* gs, const Pack<VEC>& mi, float beta, float gamma,
                                                float inv_gamma, Pack<VEC>& mn, Pack<VEC>& xn) {
-    const Pack<VEC> xi = ld_f32<VEC>(xs + (size_t)i * C + off);
+    const Pack<VEC> xi = ld_f32<VEC>(xs + i * C + off);
     float mixg[VEC], cons[VEC];
 #pragma unroll
     for (int u = 0; u < VEC; ++u) mixg[u] = cons[u] = 0.0f;
     const int p1 = t.rowptr[i + 1];
-    for (int p = t.rowptr[i]; p < p1; ++p) {
+    for (int p = t.rowptr[i]; p < p1; ++p) {  // neighbours in ascending order
         const int j = t.col[p];
         const float w = t.val[p];
-        const Pack<VEC> gj = ld_g<VEC>(gs + (size_t)j * C + off);
+        const Pack<VEC> gj = ld_g<VEC>(gs + j * C + off);
 #pragma unroll
         for (int u = 0; u < VEC; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
         if (j != i) {
-            const Pack<VEC> xj = ld_f32<VEC>(xs + (size_t)j * C + off);
+            const Pack<VEC> xj = ld_f32<VEC>(xs + j * C + off);
 #pragma unroll
             for (int u = 0; u < VEC; ++u) cons[u] = fmaf(w, xi.v[u] - xj.v[u], cons[u]);
         }
@@ -145,7 +150,7 @@ __device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, 
 template <int VEC>
 __device__ __forceinline__ void dmsgd_item(const Tables& t, int i, int off, int C, const float* ys,
                                            Pack<VEC>& xn) {
-    const Pack<VEC> yi = ld_f32<VEC>(ys + (size_t)i * C + off);
+    const Pack<VEC> yi = ld_f32<VEC>(ys + i * C + off);
     float acc[VEC];
 #pragma unroll
     for (int u = 0; u < VEC; ++u) acc[u] = 0.0f;
@@ -154,12 +159,87 @@ __device__ __forceinline__ void dmsgd_item(const Tables& t, int i, int off, int 
         const int j = t.col[p];
         if (j == i) continue;
         const float w = t.val[p];
-        const Pack<VEC> yj = ld_f32<VEC>(ys + (size_t)j * C + off);
+        const Pack<VEC> yj = ld_f32<VEC>(ys + j * C + off);
 #pragma unroll
         for (int u = 0; u < VEC; ++u) acc[u] = fmaf(w, yj.v[u] - yi.v[u], acc[u]);
     }
 #pragma unroll
     for (int u = 0; u < VEC; ++u) xn.v[u] = yi.v[u] + acc[u];
+}
+
+// Warp-cooperative variants for the pipeline kernel.  The lanes that share a row (a group of
+// G = min(32, C/4) consecutive lanes) fetch G table entries of that row with one coalesced load
+// and hand them round with shuffles, so the mixing loop has no table load on its critical
+// path.  All 32 lanes must call these together; `live` masks lanes without an item.  The
+// accumulation order (ascending neighbours, one FMA chain per column) is that of the plain
+// variants, so results are bitwise identical.
+struct RowSlot {  // one row in processing order
+    int i, p0, len;
+};
+
+template <typename GS>
+__device__ __forceinline__ void decentlam_item_coop(const int2* __restrict__ ent, RowSlot rs, int G, int off, int C,
+                                                    const float* xs, const GS* gs, const Pack<4>& mi, float beta,
+                                                    float gamma, float inv_gamma, Pack<4>& mn, Pack<4>& xn) {
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, gbase = lane & ~(G - 1), glane = lane & (G - 1);
+    const float* xcol = xs + off;
+    const GS* gcol = gs + off;
+    const Pack<4> xi = ld_f32<4>(xcol + rs.i * C);
+    float mixg[4] = {0.f, 0.f, 0.f, 0.f}, cons[4] = {0.f, 0.f, 0.f, 0.f};
+    const int len_max = __reduce_max_sync(full, rs.len);
+    for (int base = 0; base < len_max; base += G) {
+        const int idx = base + glane;
+        int2 en = make_int2(rs.i, 0);
+        if (idx < rs.len) en = ent[rs.p0 + idx];
+        const int cnt = min(G, len_max - base);
+#pragma unroll 2
+        for (int r = 0; r < cnt; ++r) {
+            const int j = __shfl_sync(full, en.x, gbase + r);
+            const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
+            if (base + r < rs.len) {
+                const Pack<4> gj = ld_g<4>(gcol + j * C);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
+                if (j != rs.i) {
+                    const Pack<4> xj = ld_f32<4>(xcol + j * C);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) cons[u] = fmaf(w, xi.v[u] - xj.v[u], cons[u]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        decentlam_finish(mixg[u], cons[u], xi.v[u], mi.v[u], beta, gamma, inv_gamma, mn.v[u], xn.v[u]);
+}
+
+__device__ __forceinline__ void dmsgd_item_coop(const int2* __restrict__ ent, RowSlot rs, int G, int off, int C,
+                                                const float* ys, Pack<4>& xn) {
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, gbase = lane & ~(G - 1), glane = lane & (G - 1);
+    const float* ycol = ys + off;
+    const Pack<4> yi = ld_f32<4>(ycol + rs.i * C);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const int len_max = __reduce_max_sync(full, rs.len);
+    for (int base = 0; base < len_max; base += G) {
+        const int idx = base + glane;
+        int2 en = make_int2(rs.i, 0);
+        if (idx < rs.len) en = ent[rs.p0 + idx];
+        const int cnt = min(G, len_max - base);
+#pragma unroll 2
+        for (int r = 0; r < cnt; ++r) {
+            const int j = __shfl_sync(full, en.x, gbase + r);
+            const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
+            if (base + r < rs.len && j != rs.i) {
+                const Pack<4> yj = ld_f32<4>(ycol + j * C);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) acc[u] = fmaf(w, yj.v[u] - yi.v[u], acc[u]);
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) xn.v[u] = yi.v[u] + acc[u];
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -182,7 +262,7 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
         const long long c_base = tile * C;
         __syncthreads();  // previous tile fully consumed (and tables staged on the first pass)
         for (int e = threadIdx.x; e < items; e += kThreads) {
-            const int i = e >> cv_shift, off = (e & cv_mask) * VEC;
+            const int i = t.order[e >> cv_shift], off = (e & cv_mask) * VEC;
             const long long c = c_base + off;
             if (c < a.d) {
                 const Pack<VEC> xi = ld_f32<VEC>(a.x + (size_t)i * a.ld + c);
@@ -202,7 +282,7 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
         }
         __syncthreads();
         for (int e = threadIdx.x; e < items; e += kThreads) {
-            const int i = e >> cv_shift, off = (e & cv_mask) * VEC;
+            const int i = t.order[e >> cv_shift], off = (e & cv_mask) * VEC;
             const long long c = c_base + off;
             if (c < a.d) {
                 Pack<VEC> xn;
@@ -271,8 +351,8 @@ struct TmaGeom {
     long long num_tiles;
 };
 
-template <int RULE, typename GT>
-__global__ void __launch_bounds__(kThreads) step_tma_kernel(const __grid_constant__ CUtensorMap tm_x,
+template <int RULE, typename GT, bool COOP>
+__global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                              const __grid_constant__ CUtensorMap tm_m,
                                                              const __grid_constant__ CUtensorMap tm_g,
                                                              dlm_step_args a, TmaGeom geo) {
@@ -307,7 +387,14 @@ __global__ void __launch_bounds__(kThreads) step_tma_kernel(const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int s = 0; s < geo.stages && s < my_tiles; ++s) issue(s, first + (long long)s * gridDim.x);
     }
-    const Tables t = stage_tables(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
+    // plain variant: tables staged in shared memory when small; cooperative variant: packed tables
+    // read from global memory (cached), one coalesced load per group of entries
+    Tables t = {a.rowptr, a.col, a.val, a.order};
+    if (!COOP) t = stage_tables(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
+    const int4* __restrict__ rows = reinterpret_cast<const int4*>(a.rows);
+    const int2* __restrict__ ent = reinterpret_cast<const int2*>(a.ent);
+    const int G = min(32, 1 << geo.cv_shift);            // lanes sharing a row
+    const int items_padded = COOP ? ((items + 31) & ~31) : items;  // whole warps take part in the shuffles
     __syncthreads();  // barriers initialised and tables staged for everyone
 
     for (long long it = 0; it < my_tiles; ++it) {
@@ -334,19 +421,19 @@ __global__ void __launch_bounds__(kThreads) step_tma_kernel(const __grid_constan
                 const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes + b * sub_x);
                 const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes + b * sub_g);
                 const long long c_base = tile_base + (long long)b * Cb;
-                for (int e = threadIdx.x; e < items; e += kThreads) {
-                    const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+                for (int e = threadIdx.x; e < items; e += blockDim.x) {
+                    const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;   // any order: purely local
                     const long long c = c_base + off;
                     if (c < a.d) {
-                        const Pack<4> xi = ld_f32<4>(xs + (size_t)i * Cb + off);
-                        const Pack<4> mi = ld_f32<4>(ms + (size_t)i * Cb + off);
-                        const Pack<4> gi = ld_g<4>(gs + (size_t)i * Cb + off);
+                        const Pack<4> xi = ld_f32<4>(xs + i * Cb + off);
+                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
+                        const Pack<4> gi = ld_g<4>(gs + i * Cb + off);
                         Pack<4> mn, y;
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], y.v[u]);
                         st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
-                        st_f32<4>(xs + (size_t)i * Cb + off, y);
+                        st_f32<4>(xs + i * Cb + off, y);
                     }
                 }
             }
@@ -357,19 +444,33 @@ __global__ void __launch_bounds__(kThreads) step_tma_kernel(const __grid_constan
             const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes + b * sub_x);
             const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes + b * sub_g);
             const long long c_base = tile_base + (long long)b * Cb;
-            for (int e = threadIdx.x; e < items; e += kThreads) {
-                const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+            for (int e = threadIdx.x; e < items_padded; e += blockDim.x) {
+                const bool live = e < items;
+                const int slot = live ? (e >> geo.cv_shift) : 0, off = (e & cv_mask) * 4;
                 const long long c = c_base + off;
-                if (c < a.d) {
-                    Pack<4> xn;
+                Pack<4> xn, mn;
+                int i;
+                if (COOP) {
+                    const int4 ri = rows[slot];
+                    i = ri.x;
                     if (RULE == DLM_RULE_DECENTLAM) {
-                        const Pack<4> mi = ld_f32<4>(ms + (size_t)i * Cb + off);
-                        Pack<4> mn;
+                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
+                        decentlam_item_coop<GT>(ent, {ri.x, ri.y, ri.z}, G, off, Cb, xs, gs, mi, a.beta, a.gamma,
+                                                a.inv_gamma, mn, xn);
+                    } else {
+                        dmsgd_item_coop(ent, {ri.x, ri.y, ri.z}, G, off, Cb, xs, xn);
+                    }
+                } else {
+                    i = t.order[slot];
+                    if (RULE == DLM_RULE_DECENTLAM) {
+                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
                         decentlam_item<4, GT>(t, i, off, Cb, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
-                        st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
                     } else {
                         dmsgd_item<4>(t, i, off, Cb, xs, xn);
                     }
+                }
+                if (live && c < a.d) {  // columns past d hold the copies' zero fill: computed, never stored
+                    if (RULE == DLM_RULE_DECENTLAM) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
                     st_f32<4>(a.x + (size_t)i * a.ld + c, xn);
                 }
             }
@@ -450,12 +551,14 @@ int ilog2(int v) {
     return l;
 }
 
-size_t table_bytes(const dlm_step_args& a) { return (size_t)(a.n + 1) * 4 + (size_t)a.nnz * 8; }
+size_t table_bytes(const dlm_step_args& a) { return (size_t)(2 * a.n + 1) * 4 + (size_t)a.nnz * 8; }
 
 int g_tune_path = 0;    // 0 auto, 1 force tile kernel, 2 force pipeline kernel (error if ineligible)
 int g_tune_cols = 0;    // tile columns, 0 = auto
 int g_tune_stages = 0;  // pipeline stages, 0 = auto
 int g_tune_ctas = 0;    // CTAs per SM, 0 = auto
+int g_tune_threads = 0;  // pipeline kernel block size (128, 256 or 512), 0 = auto
+int g_tune_coop = 0;    // 0 auto, 1 warp-cooperative mixing loop, 2 plain mixing loop
 int g_tune_tables = 0;  // 0 auto, 1 stage tables in shared memory, 2 read them from global memory
 int g_tune_tiles_per_cta = 0;  // 0 = auto; t > 0: ceil(tiles / t) CTAs; t < 0: persistent grid of sms * ctas
 
@@ -488,8 +591,8 @@ int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
 }
 
 // Returns DLM_OK if launched, DLM_ERR_UNSUPPORTED if this shape cannot use the pipeline kernel.
-template <int RULE, typename GT>
-int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
+template <int RULE, typename GT, bool COOP>
+int launch_tma_variant(const dlm_step_args& a, cudaStream_t stream) {
     const DeviceInfo& dev = device_info();
     if (!dev.ok) return DLM_ERR_CUDA;
     const bool bf16 = sizeof(GT) == 2;
@@ -498,7 +601,7 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     const size_t tab = table_bytes(a);
     // Small tables are staged in shared memory by every CTA; large ones stay in global memory
     // (all CTAs read the same few KB, so they live in L1/L2).
-    const int tables_in_smem = g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
+    const int tables_in_smem = COOP ? 0 : g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
     const size_t fixed = 128 + kMaxStages * 8 + 16 + (tables_in_smem ? tab : 0);
     const size_t budget = (size_t)dev.smem_optin;
     auto stage_bytes_for = [&](int C, uint32_t& xb, uint32_t& gb) {
@@ -547,14 +650,24 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     geo.tables_in_smem = tables_in_smem;
     geo.num_tiles = (a.d + C - 1) / C;
     size_t smem = fixed + (size_t)stages * sb;
-    auto kern = step_tma_kernel<RULE, GT>;
+    auto kern = step_tma_kernel<RULE, GT, COOP>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DLM_ERR_CUDA;
     long long grid = tiles_per_cta > 0 ? (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta
                                        : std::min<long long>(geo.num_tiles, (long long)dev.sms * ctas);
-    kern<<<(unsigned)grid, kThreads, smem, stream>>>(tm_x, tm_m, tm_g, a, geo);
+    // long neighbour lists need more warps in flight to hide the mixing loop's latency
+    const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512)
+                            ? g_tune_threads : (a.max_degree > 8 ? 512 : 256);
+    kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_m, tm_g, a, geo);
     dlm_count_launch(1);
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
+
+// Plain mixing loop for very sparse rows, warp-cooperative table fetch otherwise.
+template <int RULE, typename GT>
+int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
+    const bool coop = g_tune_coop == 1 ? true : g_tune_coop == 2 ? false : a.max_degree > 8;
+    return coop ? launch_tma_variant<RULE, GT, true>(a, stream) : launch_tma_variant<RULE, GT, false>(a, stream);
 }
 
 template <int RULE, typename GT>
@@ -616,6 +729,8 @@ DLM_API int dlm_set_tuning(int knob, int value) {
     case 3: g_tune_ctas = value; return DLM_OK;
     case 4: g_tune_tiles_per_cta = value; return DLM_OK;
     case 5: g_tune_tables = value; return DLM_OK;
+    case 6: g_tune_threads = value; return DLM_OK;
+    case 7: g_tune_coop = value; return DLM_OK;
     default: return DLM_ERR_KIND;
     }
 }

@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 #include <new>
 
 #include "dlm_internal.h"
@@ -58,9 +59,42 @@ std::vector<Edge> unique_neighbours(int i, const std::vector<int32_t>& js, int q
     return nb;
 }
 
+// Processing order for the kernels: rows of similar length next to each other, so that the rows
+// sharing a warp run the same number of neighbour iterations.
+void make_order(dlm_slot& s) {
+    const int n = (int)s.rowptr.size() - 1;
+    s.order.resize(n);
+    for (int i = 0; i < n; ++i) s.order[i] = i;
+    std::stable_sort(s.order.begin(), s.order.end(), [&](int32_t a, int32_t b) {
+        return s.rowptr[a + 1] - s.rowptr[a] > s.rowptr[b + 1] - s.rowptr[b];
+    });
+    s.rows.resize((size_t)4 * n);
+    for (int r = 0; r < n; ++r) {
+        const int i = s.order[r];
+        s.rows[4 * r + 0] = i;
+        s.rows[4 * r + 1] = s.rowptr[i];
+        s.rows[4 * r + 2] = s.rowptr[i + 1] - s.rowptr[i];
+        s.rows[4 * r + 3] = 0;
+    }
+    s.ent.resize(2 * s.col.size());
+    for (size_t p = 0; p < s.col.size(); ++p) {
+        s.ent[2 * p] = s.col[p];
+        std::memcpy(&s.ent[2 * p + 1], &s.val[p], sizeof(float));
+    }
+}
+
 int upload(dlm_slot& s) {
     size_t nr = s.rowptr.size() * sizeof(int32_t), nc = s.col.size() * sizeof(int32_t),
            nv = s.val.size() * sizeof(float);
+    if (cudaMalloc((void**)&s.d_rows, s.rows.size() * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMalloc((void**)&s.d_ent, std::max<size_t>(1, s.ent.size()) * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_rows, s.rows.data(), s.rows.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_ent, s.ent.data(), s.ent.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    if (cudaMalloc((void**)&s.d_order, s.order.size() * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_order, s.order.data(), s.order.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return DLM_ERR_CUDA;
     if (cudaMalloc((void**)&s.d_rowptr, nr) != cudaSuccess) return DLM_ERR_CUDA;
     if (cudaMalloc((void**)&s.d_col, nc) != cudaSuccess) return DLM_ERR_CUDA;
     if (cudaMalloc((void**)&s.d_val, nv) != cudaSuccess) return DLM_ERR_CUDA;
@@ -181,6 +215,7 @@ int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, c
         }
         }
     }
+    for (int slot = 0; slot < period && rc == DLM_OK; ++slot) make_order(t->slots[slot]);
     // Without a CUDA device the handle stays host-only (tables can be inspected, steps fail).
     int ndev = 0;
     bool have_device = rc == DLM_OK && cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0;
@@ -235,6 +270,9 @@ int topology_tables_device(const dlm_topology* topo, int slot, const int32_t** r
 int topology_destroy(dlm_topology* topo) {
     if (!topo) return DLM_OK;
     for (dlm_slot& s : topo->slots) {
+        if (s.d_order) cudaFree(s.d_order);
+        if (s.d_rows) cudaFree(s.d_rows);
+        if (s.d_ent) cudaFree(s.d_ent);
         if (s.d_rowptr) cudaFree(s.d_rowptr);
         if (s.d_col) cudaFree(s.d_col);
         if (s.d_val) cudaFree(s.d_val);

@@ -108,18 +108,20 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
     """The plain-load kernel and the bulk-copy pipeline kernel round identically."""
     from paper_2104_11981_b200 import binding as B
     dev = torch.device("cuda:0")
-    n, d = 16, 100_000
-    topo, _ = build_both("static_exp", n)
+    n, d = 24, 100_000                       # 24 rows: the last warp of a tile is partly idle
+    topo, _ = build_both("er_mh", n, graph_seed=9, er_p=0.5)     # rows of very different lengths
     gt = torch.bfloat16 if g_dtype == "bf16" else torch.float32
     x0 = inputs.normal_torch((n, d), 0.02, 1, dev); m0 = inputs.normal_torch((n, d), 0.01, 2, dev)
     g = inputs.normal_torch((n, d), 1e-3, 3, dev, dtype=gt)
     outs = []
     try:
-        # (path, tile columns, stages, tiles per CTA, tables)
-        for path, cols, stages, tpc, tab in ((1, 0, 0, 0, 0), (2, 0, 0, 0, 0), (2, 64, 2, -1, 1), (2, 256, 3, -1, 2),
-                                             (2, 512, 2, 4, 0), (2, 32, 1, 3, 2), (1, 128, 0, 0, 0)):
+        # (path, tile columns, stages, tiles per CTA, tables, threads, mixing loop)
+        for path, cols, stages, tpc, tab, thr, coop in ((1, 0, 0, 0, 0, 0, 0), (2, 0, 0, 0, 0, 0, 0),
+                                                        (2, 64, 2, -1, 1, 0, 2), (2, 256, 3, -1, 2, 512, 1),
+                                                        (2, 512, 2, 4, 0, 128, 2), (2, 32, 1, 3, 2, 512, 1),
+                                                        (2, 8, 1, 1, 0, 256, 1), (1, 128, 0, 0, 0, 0, 0)):
             B.set_tuning(0, path); B.set_tuning(1, cols); B.set_tuning(2, stages)
-            B.set_tuning(4, tpc); B.set_tuning(5, tab)
+            B.set_tuning(4, tpc); B.set_tuning(5, tab); B.set_tuning(6, thr); B.set_tuning(7, coop)
             x, m = x0.clone(), m0.clone()
             for k in range(3):
                 lib_rule(rule, topo, k, x, m, g, 0.9, 0.1)
@@ -127,7 +129,7 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
             assert B.kernel_error() == 0
             outs.append((x, m))
     finally:
-        for knob in range(6):
+        for knob in range(8):
             B.set_tuning(knob, 0)
     for x, m in outs[1:]:
         assert torch.equal(x, outs[0][0]) and torch.equal(m, outs[0][1])
