@@ -719,6 +719,10 @@ int dlm_launch_step(int rule, const dlm_step_args& a, void* stream) {
                                    : launch_rule<DLM_RULE_DMSGD, float>(a, s);
 }
 
+extern int g_lsq_tune_splits;
+extern int g_lsq_tune_bulk;
+int dlm_lsq_take_error(int* flag);
+
 extern "C" {
 
 DLM_API int dlm_set_tuning(int knob, int value) {
@@ -731,6 +735,8 @@ DLM_API int dlm_set_tuning(int knob, int value) {
     case 5: g_tune_tables = value; return DLM_OK;
     case 6: g_tune_threads = value; return DLM_OK;
     case 7: g_tune_coop = value; return DLM_OK;
+    case 8: g_lsq_tune_splits = value; return DLM_OK;
+    case 9: g_lsq_tune_bulk = value; return DLM_OK;
     default: return DLM_ERR_KIND;
     }
 }
@@ -743,7 +749,10 @@ DLM_API int dlm_kernel_error(int* flag) {
         int zero = 0;
         if (cudaMemcpyToSymbol(g_kernel_error, &zero, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
     }
-    *flag = v;
+    int lsq = 0;
+    int rc = dlm_lsq_take_error(&lsq);
+    if (rc != DLM_OK) return rc;
+    *flag = v != 0 ? v : lsq;
     return DLM_OK;
 }
 
