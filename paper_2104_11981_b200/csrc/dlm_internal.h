@@ -11,7 +11,7 @@ struct dlm_slot {
     std::vector<float> val;
     std::vector<int32_t> order;  // rows sorted by decreasing degree (stable): the kernels' processing order
     int32_t* d_order = nullptr;
-    // packed copies for the warp-cooperative kernels: rows[r] = {i, first entry, length, 0} in
+    // packed copies for the warp-cooperative kernels: rows[r] = {i, first entry, length, bits of S_i = sum_j w_ij} in
     // processing order; ent[p] = {col[p], bits of val[p]}
     std::vector<int32_t> rows, ent;
     int32_t* d_rows = nullptr;
@@ -43,7 +43,7 @@ struct dlm_step_args {
     const int32_t* col;     // device
     const float* val;       // device
     const int32_t* order;   // device, row processing order (a permutation of 0..n-1)
-    const int32_t* rows;    // device, int4 per row in processing order {i, first entry, length, 0}
+    const int32_t* rows;    // device, int4 per row in processing order {i, first entry, length, bits of S_i}
     const int32_t* ent;     // device, int2 per entry {col, bits of val}
     int nnz;
     int max_degree;

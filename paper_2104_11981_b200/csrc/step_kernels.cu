@@ -484,6 +484,167 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Merged-staging DecentLaM kernel for long neighbour lists (many nodes, dense rows).
+//
+// With z_j = x_j - r (r = row 0's value of the column: a common reference that keeps z small
+// whenever the replicas are close) and v_j = g_j - z_j / gamma, Eq. (decentLaM-x-1) reads
+//     g~_i = sum_{j in N_i} w_ij v_j + z_i S_i / gamma,      S_i = sum_{j != i} w_ij + w_ii (stored),
+// (expand: sum_j w_ij g_j + (1/gamma) sum_{j != i} w_ij (z_i - z_j); the self term of the v-sum
+// cancels against w_ii z_i / gamma).  So ONE staged value per neighbour, no subtraction and no
+// self special case in the loop.  Pass 1 turns the staged (x, g) into v: in place of g for fp32
+// gradients, in a tile of its own for bf16.  Pass 2: a thread owns two float4 column groups of a
+// row, the L = C/8 lanes that share the row fetch its table entries together and hand them round
+// with shuffles; slots past the end of a row carry weight 0 and point at row i itself, so the
+// loop is branch-free.  m is not staged: each thread reads its own m from global memory while
+// the loop runs.  Tables live in shared memory when they fit (the large shared-memory carve-out
+// leaves too little L1 to keep them cached otherwise).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(addr)
+                 : "memory");
+    return v;
+}
+
+struct MergedGeom {
+    int C;          // tile columns (power of two, 32 .. 256)
+    int cv_shift;   // log2(C / 4)
+    int tables_in_smem;
+    uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
+    uint32_t v_off, g_off; // byte offsets of the v tile and of the g landing area inside the stage
+    uint32_t stage_bytes;
+    uint32_t tx_bytes;
+    long long num_tiles;
+};
+
+template <typename GT>
+__global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant__ CUtensorMap tm_x,
+                                                           const __grid_constant__ CUtensorMap tm_g,
+                                                           dlm_step_args a, MergedGeom geo) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned char* st = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
+    uint64_t* bar_ptr = reinterpret_cast<uint64_t*>(st + geo.stage_bytes);
+    int4* s_rows = reinterpret_cast<int4*>(st + geo.stage_bytes + 16);
+    int2* s_ent = reinterpret_cast<int2*>(s_rows + a.n);
+    const uint32_t bar = smem_u32(bar_ptr);
+
+    const long long first = blockIdx.x;
+    const long long my_tiles = first < geo.num_tiles ? (geo.num_tiles - first + gridDim.x - 1) / gridDim.x : 0;
+    const int C = geo.C;
+    auto issue = [&](long long tile) {
+        const int c0 = (int)(tile * C);
+        mbar_expect_tx(bar, geo.tx_bytes);
+        tma_load_2d(smem_u32(st), &tm_x, c0, 0, bar);
+        tma_load_2d(smem_u32(st + geo.g_off), &tm_g, c0, 0, bar);
+    };
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (my_tiles > 0) issue(first);
+    }
+    const int4* rows = reinterpret_cast<const int4*>(a.rows);
+    const int2* ent = reinterpret_cast<const int2*>(a.ent);
+    if (geo.tables_in_smem) {  // overlaps the first copies
+        for (int r = threadIdx.x; r < a.n; r += blockDim.x) s_rows[r] = rows[r];
+        for (int p = threadIdx.x; p < a.nnz; p += blockDim.x) s_ent[p] = ent[p];
+        rows = s_rows;
+        ent = s_ent;
+    }
+    __syncthreads();
+
+    const float* xs = reinterpret_cast<const float*>(st);
+    float* vs = reinterpret_cast<float*>(st + geo.v_off);
+    const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off);
+    const int items = a.n << geo.cv_shift;
+    const int cv_mask = (1 << geo.cv_shift) - 1;
+    const unsigned full = 0xffffffffu;
+    const int lshift = geo.cv_shift - 1, L = 1 << lshift;  // lanes per row in pass 2
+    const int witems = a.n << lshift, witems_padded = (witems + 31) & ~31;
+    const int lane = threadIdx.x & 31, gbase = lane & ~(L - 1), glane = lane & (L - 1);
+    const uint32_t row_bytes = (uint32_t)C * 4;
+
+    for (long long it = 0; it < my_tiles; ++it) {
+        const bool arrived = mbar_wait(bar, (uint32_t)(it & 1));
+        if (!__syncthreads_and(arrived)) {  // uniform decision: give up together
+            if (threadIdx.x == 0) atomicExch(&g_kernel_error, 3);
+            return;                          // single stage: no other copy of this CTA is in flight
+        }
+        const long long tile_base = (first + it * gridDim.x) * C;
+        // pass 1: v = g - (x - r) / gamma
+        for (int e = threadIdx.x; e < items; e += blockDim.x) {
+            const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+            const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
+            const Pack<4> gi = ld_g<4>(gs + i * C + off);
+            Pack<4> v;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
+            st_f32<4>(vs + i * C + off, v);
+        }
+        __syncthreads();
+        // pass 2
+        for (int e = threadIdx.x; e < witems_padded; e += blockDim.x) {
+            const bool live = e < witems;
+            const int4 ri = rows[live ? (e >> lshift) : 0];
+            const int i = ri.x, len = ri.z;
+            // column groups {q, q + L}; with four lanes per row, neighbouring rows take the two
+            // halves in opposite order so that a quarter warp still covers all 32 banks
+            const int par = (L == 4) ? ((e >> lshift) & 1) : 0;
+            const int off0 = (L == 4 ? glane + 4 * par : glane) * 4;
+            const int off1 = (L == 4 ? glane + 4 * (1 - par) : glane + L) * 4;
+            const long long c0 = tile_base + off0, c1 = tile_base + off1;
+            const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;
+            Pack<4> m0 = {{0.f, 0.f, 0.f, 0.f}}, m1 = {{0.f, 0.f, 0.f, 0.f}};
+            if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
+            if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t vb0 = smem_u32(vs) + off0 * 4, vb1 = smem_u32(vs) + off1 * 4;
+            const int len_max = __reduce_max_sync(full, len);
+            for (int base0 = 0; base0 < len_max; base0 += L) {
+                int2 en = make_int2(i, 0);  // filler: adds exactly 0 * v_i
+                if (base0 + glane < len) en = ent[ri.y + base0 + glane];
+                const int cnt = min(L, (len_max - base0 + 3) & ~3);
+#pragma unroll 4
+                for (int r = 0; r < cnt; ++r) {
+                    const int j = __shfl_sync(full, en.x, gbase + r);
+                    const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
+                    const float4 v0 = lds128(vb0 + (uint32_t)j * row_bytes);
+                    const float4 v1 = lds128(vb1 + (uint32_t)j * row_bytes);
+                    acc0[0] = fmaf(w, v0.x, acc0[0]); acc0[1] = fmaf(w, v0.y, acc0[1]);
+                    acc0[2] = fmaf(w, v0.z, acc0[2]); acc0[3] = fmaf(w, v0.w, acc0[3]);
+                    acc1[0] = fmaf(w, v1.x, acc1[0]); acc1[1] = fmaf(w, v1.y, acc1[1]);
+                    acc1[2] = fmaf(w, v1.z, acc1[2]); acc1[3] = fmaf(w, v1.w, acc1[3]);
+                }
+            }
+            const float S_i = __int_as_float(ri.w);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int off = h ? off1 : off0;
+                const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
+                Pack<4> mn, xn;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, h ? acc1[u] : acc0[u]);
+                    mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
+                    xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
+                }
+                if (h ? st1 : st0) {
+                    st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
+                    st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
+                }
+            }
+        }
+        if (it + 1 < my_tiles) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();
+            if (threadIdx.x == 0) issue(first + (it + 1) * gridDim.x);
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
@@ -558,7 +719,7 @@ int g_tune_cols = 0;    // tile columns, 0 = auto
 int g_tune_stages = 0;  // pipeline stages, 0 = auto
 int g_tune_ctas = 0;    // CTAs per SM, 0 = auto
 int g_tune_threads = 0;  // pipeline kernel block size (128, 256 or 512), 0 = auto
-int g_tune_coop = 0;    // 0 auto, 1 warp-cooperative mixing loop, 2 plain mixing loop
+int g_tune_coop = 0;    // 0 auto, 1 warp-cooperative mixing loop, 2 plain mixing loop, 3 merged-staging kernel
 int g_tune_tables = 0;  // 0 auto, 1 stage tables in shared memory, 2 read them from global memory
 int g_tune_tiles_per_cta = 0;  // 0 = auto; t > 0: ceil(tiles / t) CTAs; t < 0: persistent grid of sms * ctas
 
@@ -663,11 +824,65 @@ int launch_tma_variant(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// Plain mixing loop for very sparse rows, warp-cooperative table fetch otherwise.
+// DecentLaM with merged staging (long rows).  DLM_ERR_UNSUPPORTED if the shape does not fit.
+template <typename GT>
+int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return DLM_ERR_CUDA;
+    const bool bf16 = sizeof(GT) == 2;
+    if (a.n > 256 || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
+    int C = 1 << ilog2(std::max(1, (int)(32768 / ((size_t)a.n * 4))));
+    C = std::max(32, std::min(256, C));
+    if (g_tune_cols >= 32 && g_tune_cols <= 256 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
+    const size_t tab = (size_t)a.n * 16 + (size_t)a.nnz * 8;
+    MergedGeom geo;
+    size_t smem = 0;
+    for (;; C /= 2) {
+        if (C < 32) return DLM_ERR_UNSUPPORTED;
+        const size_t xb = ((size_t)a.n * C * 4 + 127) & ~(size_t)127;
+        const size_t gb = ((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127;
+        geo.x_bytes = (uint32_t)xb;
+        geo.v_off = (uint32_t)xb;                       // fp32: v overwrites g in place
+        geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);     // bf16: g lands behind the v tile
+        geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
+        // tables in shared memory if two CTAs per SM still fit, or if one CTA fits and they are large
+        const size_t fixed = 128 + 16 + 16;
+        const size_t with_tab = fixed + geo.stage_bytes + tab;
+        geo.tables_in_smem = g_tune_tables == 2 ? 0 : (with_tab <= (size_t)dev.smem_optin / 2 - 1024 || g_tune_tables == 1);
+        smem = geo.tables_in_smem ? with_tab : fixed + geo.stage_bytes;
+        if (smem <= (size_t)dev.smem_optin / 2 - 1024 || (C == 32 && smem <= (size_t)dev.smem_optin)) break;
+    }
+    geo.C = C;
+    geo.cv_shift = ilog2(C / 4);
+    geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
+    geo.num_tiles = (a.d + C - 1) / C;
+    CUtensorMap tm_x, tm_g;
+    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, C) || !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, C))
+        return DLM_ERR_UNSUPPORTED;
+    auto kern = step_merged_kernel<GT>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : (geo.tables_in_smem ? 8 : 4);
+    const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512) ? g_tune_threads : 512;
+    kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_g, a, geo);
+    dlm_count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
+
+// Plain mixing loop for sparse rows, warp-cooperative table fetch for long rows; DecentLaM on
+// long rows takes the merged-staging kernel when the shape allows it.
 template <int RULE, typename GT>
 int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
-    const bool coop = g_tune_coop == 1 ? true : g_tune_coop == 2 ? false : a.max_degree > 8;
-    return coop ? launch_tma_variant<RULE, GT, true>(a, stream) : launch_tma_variant<RULE, GT, false>(a, stream);
+    // measured on B200 at n = 256: rows of up to 9 entries run fastest with the cooperative loop,
+    // rows of ~14 (up to 23) entries with merged staging
+    const int mode = g_tune_coop == 1 ? 1 : g_tune_coop == 2 ? 0 : g_tune_coop == 3 ? 2
+                     : (a.max_degree >= 12 ? 2 : a.max_degree > 8 ? 1 : 0);
+    if (mode == 2 && RULE == DLM_RULE_DECENTLAM) {
+        int rc = launch_merged<GT>(a, stream);
+        if (rc != DLM_ERR_UNSUPPORTED) return rc;
+    }
+    return mode >= 1 ? launch_tma_variant<RULE, GT, true>(a, stream) : launch_tma_variant<RULE, GT, false>(a, stream);
 }
 
 template <int RULE, typename GT>

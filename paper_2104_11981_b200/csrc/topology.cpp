@@ -74,7 +74,10 @@ void make_order(dlm_slot& s) {
         s.rows[4 * r + 0] = i;
         s.rows[4 * r + 1] = s.rowptr[i];
         s.rows[4 * r + 2] = s.rowptr[i + 1] - s.rowptr[i];
-        s.rows[4 * r + 3] = 0;
+        double row_sum = 0.0;  // S_i = sum_j w_ij over the stored weights, rounded once
+        for (int32_t p = s.rowptr[i]; p < s.rowptr[i + 1]; ++p) row_sum += (double)s.val[p];
+        const float S_i = (float)row_sum;
+        std::memcpy(&s.rows[4 * r + 3], &S_i, sizeof(float));
     }
     s.ent.resize(2 * s.col.size());
     for (size_t p = 0; p < s.col.size(); ++p) {
