@@ -45,6 +45,33 @@ def parse_args():
     return ap.parse_args()
 
 
+# DRAM counters of step_tma_kernel<DecentLaM, fp32 g> from the ncu capture summarised in
+# profiles/step_tma_kernel_decentlam_n16_d2M.md (n = 16, 2,097,152 columns), per node-parameter.
+# Valid only for the kernel source they were taken from: reported while the source file's
+# SHA-256 matches, otherwise "traffic" is null.
+NCU_CAPTURE = {
+    "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
+    "sha256": "f28533ba5eb2cf9b88f328d927d52440c287b2d5dfe5bb8c9568e3864ef0b0cc",
+    "workload": "cfg2",
+    "dram_read_bytes_per_np": 402.70e6 / (16 * 2097152),
+    "dram_write_bytes_per_np": 216.02e6 / (16 * 2097152),
+}
+
+
+def ncu_traffic(workload, units):
+    """DRAM bytes per launch scaled from the small-case capture by the units processed, or None."""
+    import hashlib
+    if workload != NCU_CAPTURE["workload"]:
+        return None
+    try:
+        with open(os.path.join(ROOT, NCU_CAPTURE["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != NCU_CAPTURE["sha256"]:
+                return None
+    except OSError:
+        return None
+    return (NCU_CAPTURE["dram_read_bytes_per_np"] + NCU_CAPTURE["dram_write_bytes_per_np"]) * units
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -326,7 +353,7 @@ def run_ours(args):
                        "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": f"working set {(8 + g.element_size()) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": f"of {peak_kind}",
+                         "traffic": ncu_traffic(args.workload, n * d), "peak_kind": f"of {peak_kind}",
                          "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "cpu_baseline": cpu_baseline,
             "other_rules": extra,
