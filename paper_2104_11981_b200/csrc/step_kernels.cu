@@ -167,81 +167,6 @@ __device__ __forceinline__ void dmsgd_item(const Tables& t, int i, int off, int 
     for (int u = 0; u < VEC; ++u) xn.v[u] = yi.v[u] + acc[u];
 }
 
-// Warp-cooperative variants for the pipeline kernel.  The lanes that share a row (a group of
-// G = min(32, C/4) consecutive lanes) fetch G table entries of that row with one coalesced load
-// and hand them round with shuffles, so the mixing loop has no table load on its critical
-// path.  All 32 lanes must call these together; `live` masks lanes without an item.  The
-// accumulation order (ascending neighbours, one FMA chain per column) is that of the plain
-// variants, so results are bitwise identical.
-struct RowSlot {  // one row in processing order
-    int i, p0, len;
-};
-
-template <typename GS>
-__device__ __forceinline__ void decentlam_item_coop(const int2* __restrict__ ent, RowSlot rs, int G, int off, int C,
-                                                    const float* xs, const GS* gs, const Pack<4>& mi, float beta,
-                                                    float gamma, float inv_gamma, Pack<4>& mn, Pack<4>& xn) {
-    const unsigned full = 0xffffffffu;
-    const int lane = threadIdx.x & 31, gbase = lane & ~(G - 1), glane = lane & (G - 1);
-    const float* xcol = xs + off;
-    const GS* gcol = gs + off;
-    const Pack<4> xi = ld_f32<4>(xcol + rs.i * C);
-    float mixg[4] = {0.f, 0.f, 0.f, 0.f}, cons[4] = {0.f, 0.f, 0.f, 0.f};
-    const int len_max = __reduce_max_sync(full, rs.len);
-    for (int base = 0; base < len_max; base += G) {
-        const int idx = base + glane;
-        int2 en = make_int2(rs.i, 0);
-        if (idx < rs.len) en = ent[rs.p0 + idx];
-        const int cnt = min(G, len_max - base);
-#pragma unroll 2
-        for (int r = 0; r < cnt; ++r) {
-            const int j = __shfl_sync(full, en.x, gbase + r);
-            const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
-            if (base + r < rs.len) {
-                const Pack<4> gj = ld_g<4>(gcol + j * C);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
-                if (j != rs.i) {
-                    const Pack<4> xj = ld_f32<4>(xcol + j * C);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) cons[u] = fmaf(w, xi.v[u] - xj.v[u], cons[u]);
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-        decentlam_finish(mixg[u], cons[u], xi.v[u], mi.v[u], beta, gamma, inv_gamma, mn.v[u], xn.v[u]);
-}
-
-__device__ __forceinline__ void dmsgd_item_coop(const int2* __restrict__ ent, RowSlot rs, int G, int off, int C,
-                                                const float* ys, Pack<4>& xn) {
-    const unsigned full = 0xffffffffu;
-    const int lane = threadIdx.x & 31, gbase = lane & ~(G - 1), glane = lane & (G - 1);
-    const float* ycol = ys + off;
-    const Pack<4> yi = ld_f32<4>(ycol + rs.i * C);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int len_max = __reduce_max_sync(full, rs.len);
-    for (int base = 0; base < len_max; base += G) {
-        const int idx = base + glane;
-        int2 en = make_int2(rs.i, 0);
-        if (idx < rs.len) en = ent[rs.p0 + idx];
-        const int cnt = min(G, len_max - base);
-#pragma unroll 2
-        for (int r = 0; r < cnt; ++r) {
-            const int j = __shfl_sync(full, en.x, gbase + r);
-            const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
-            if (base + r < rs.len && j != rs.i) {
-                const Pack<4> yj = ld_f32<4>(ycol + j * C);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) acc[u] = fmaf(w, yj.v[u] - yi.v[u], acc[u]);
-            }
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) xn.v[u] = yi.v[u] + acc[u];
-}
-
 // ---------------------------------------------------------------------------------------------
 // Plain-load tile kernel (any alignment).  C is a power of two multiple of VEC.
 // Shared memory: xs[n*C] fp32 (x, or y for DmSGD) | gs[n*C] fp32 (DecentLaM only) | tables.
@@ -351,7 +276,7 @@ struct TmaGeom {
     long long num_tiles;
 };
 
-template <int RULE, typename GT, bool COOP>
+template <int RULE, typename GT>
 __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                              const __grid_constant__ CUtensorMap tm_m,
                                                              const __grid_constant__ CUtensorMap tm_g,
@@ -387,14 +312,8 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int s = 0; s < geo.stages && s < my_tiles; ++s) issue(s, first + (long long)s * gridDim.x);
     }
-    // plain variant: tables staged in shared memory when small; cooperative variant: packed tables
-    // read from global memory (cached), one coalesced load per group of entries
-    Tables t = {a.rowptr, a.col, a.val, a.order};
-    if (!COOP) t = stage_tables(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
-    const int4* __restrict__ rows = reinterpret_cast<const int4*>(a.rows);
-    const int2* __restrict__ ent = reinterpret_cast<const int2*>(a.ent);
-    const int G = min(32, 1 << geo.cv_shift);            // lanes sharing a row
-    const int items_padded = COOP ? ((items + 31) & ~31) : items;  // whole warps take part in the shuffles
+    // tables staged in shared memory when small, else read from global memory (cached)
+    const Tables t = stage_tables(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
     __syncthreads();  // barriers initialised and tables staged for everyone
 
     for (long long it = 0; it < my_tiles; ++it) {
@@ -444,33 +363,19 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
             const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes + b * sub_x);
             const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes + b * sub_g);
             const long long c_base = tile_base + (long long)b * Cb;
-            for (int e = threadIdx.x; e < items_padded; e += blockDim.x) {
-                const bool live = e < items;
-                const int slot = live ? (e >> geo.cv_shift) : 0, off = (e & cv_mask) * 4;
+            for (int e = threadIdx.x; e < items; e += blockDim.x) {
+                const int i = t.order[e >> geo.cv_shift], off = (e & cv_mask) * 4;
                 const long long c = c_base + off;
-                Pack<4> xn, mn;
-                int i;
-                if (COOP) {
-                    const int4 ri = rows[slot];
-                    i = ri.x;
+                if (c < a.d) {  // columns past d hold the copies' zero fill
+                    Pack<4> xn;
                     if (RULE == DLM_RULE_DECENTLAM) {
                         const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
-                        decentlam_item_coop<GT>(ent, {ri.x, ri.y, ri.z}, G, off, Cb, xs, gs, mi, a.beta, a.gamma,
-                                                a.inv_gamma, mn, xn);
-                    } else {
-                        dmsgd_item_coop(ent, {ri.x, ri.y, ri.z}, G, off, Cb, xs, xn);
-                    }
-                } else {
-                    i = t.order[slot];
-                    if (RULE == DLM_RULE_DECENTLAM) {
-                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
+                        Pack<4> mn;
                         decentlam_item<4, GT>(t, i, off, Cb, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
+                        st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
                     } else {
                         dmsgd_item<4>(t, i, off, Cb, xs, xn);
                     }
-                }
-                if (live && c < a.d) {  // columns past d hold the copies' zero fill: computed, never stored
-                    if (RULE == DLM_RULE_DECENTLAM) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
                     st_f32<4>(a.x + (size_t)i * a.ld + c, xn);
                 }
             }
@@ -719,7 +624,7 @@ int g_tune_cols = 0;    // tile columns, 0 = auto
 int g_tune_stages = 0;  // pipeline stages, 0 = auto
 int g_tune_ctas = 0;    // CTAs per SM, 0 = auto
 int g_tune_threads = 0;  // pipeline kernel block size (128, 256 or 512), 0 = auto
-int g_tune_coop = 0;    // 0 auto, 1 warp-cooperative mixing loop, 2 plain mixing loop, 3 merged-staging kernel
+int g_tune_mix = 0;     // 0 auto, 1 pipeline kernel with the plain mixing loop, 2 merged-staging kernel
 int g_tune_tables = 0;  // 0 auto, 1 stage tables in shared memory, 2 read them from global memory
 int g_tune_tiles_per_cta = 0;  // 0 = auto; t > 0: ceil(tiles / t) CTAs; t < 0: persistent grid of sms * ctas
 
@@ -752,8 +657,8 @@ int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
 }
 
 // Returns DLM_OK if launched, DLM_ERR_UNSUPPORTED if this shape cannot use the pipeline kernel.
-template <int RULE, typename GT, bool COOP>
-int launch_tma_variant(const dlm_step_args& a, cudaStream_t stream) {
+template <int RULE, typename GT>
+int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     const DeviceInfo& dev = device_info();
     if (!dev.ok) return DLM_ERR_CUDA;
     const bool bf16 = sizeof(GT) == 2;
@@ -762,7 +667,7 @@ int launch_tma_variant(const dlm_step_args& a, cudaStream_t stream) {
     const size_t tab = table_bytes(a);
     // Small tables are staged in shared memory by every CTA; large ones stay in global memory
     // (all CTAs read the same few KB, so they live in L1/L2).
-    const int tables_in_smem = COOP ? 0 : g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
+    const int tables_in_smem = g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
     const size_t fixed = 128 + kMaxStages * 8 + 16 + (tables_in_smem ? tab : 0);
     const size_t budget = (size_t)dev.smem_optin;
     auto stage_bytes_for = [&](int C, uint32_t& xb, uint32_t& gb) {
@@ -811,7 +716,7 @@ int launch_tma_variant(const dlm_step_args& a, cudaStream_t stream) {
     geo.tables_in_smem = tables_in_smem;
     geo.num_tiles = (a.d + C - 1) / C;
     size_t smem = fixed + (size_t)stages * sb;
-    auto kern = step_tma_kernel<RULE, GT, COOP>;
+    auto kern = step_tma_kernel<RULE, GT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DLM_ERR_CUDA;
     long long grid = tiles_per_cta > 0 ? (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta
@@ -870,19 +775,17 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// Plain mixing loop for sparse rows, warp-cooperative table fetch for long rows; DecentLaM on
-// long rows takes the merged-staging kernel when the shape allows it.
+// DecentLaM on rows of 12 or more entries takes the merged-staging kernel when the shape allows
+// it (measured on B200 at n = 256: 9-entry rows are faster with the plain loop, ~14-entry rows with
+// merged staging); everything else the pipeline kernel with the plain mixing loop.
 template <int RULE, typename GT>
 int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
-    // measured on B200 at n = 256: rows of up to 9 entries run fastest with the cooperative loop,
-    // rows of ~14 (up to 23) entries with merged staging
-    const int mode = g_tune_coop == 1 ? 1 : g_tune_coop == 2 ? 0 : g_tune_coop == 3 ? 2
-                     : (a.max_degree >= 12 ? 2 : a.max_degree > 8 ? 1 : 0);
-    if (mode == 2 && RULE == DLM_RULE_DECENTLAM) {
+    const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : a.max_degree >= 12;
+    if (merged && RULE == DLM_RULE_DECENTLAM) {
         int rc = launch_merged<GT>(a, stream);
         if (rc != DLM_ERR_UNSUPPORTED) return rc;
     }
-    return mode >= 1 ? launch_tma_variant<RULE, GT, true>(a, stream) : launch_tma_variant<RULE, GT, false>(a, stream);
+    return launch_tma_plain<RULE, GT>(a, stream);
 }
 
 template <int RULE, typename GT>
@@ -949,7 +852,7 @@ DLM_API int dlm_set_tuning(int knob, int value) {
     case 4: g_tune_tiles_per_cta = value; return DLM_OK;
     case 5: g_tune_tables = value; return DLM_OK;
     case 6: g_tune_threads = value; return DLM_OK;
-    case 7: g_tune_coop = value; return DLM_OK;
+    case 7: g_tune_mix = value; return DLM_OK;
     case 8: g_lsq_tune_splits = value; return DLM_OK;
     case 9: g_lsq_tune_bulk = value; return DLM_OK;
     default: return DLM_ERR_KIND;

@@ -117,18 +117,18 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
     try:
         # (path, tile columns, stages, tiles per CTA, tables, threads, mixing loop); the rows of this
         # graph are long, so "mixing loop 0" (automatic) picks the merged-staging kernel on path 2
-        variants = ((1, 0, 0, 0, 0, 0, 0), (2, 0, 0, 0, 0, 0, 1), (2, 64, 2, -1, 1, 0, 2), (2, 256, 3, -1, 2, 512, 1),
-                    (2, 512, 2, 4, 0, 128, 2), (2, 32, 1, 3, 2, 512, 1), (2, 8, 1, 1, 0, 256, 1), (1, 128, 0, 0, 0, 0, 0),
-                    (2, 0, 0, 0, 0, 0, 0), (2, 32, 0, 2, 0, 128, 3), (2, 64, 0, 1, 2, 512, 3), (2, 256, 0, 0, 1, 256, 3))
-        for path, cols, stages, tpc, tab, thr, coop in variants:
+        variants = ((1, 0, 0, 0, 0, 0, 0), (2, 0, 0, 0, 0, 0, 1), (2, 64, 2, -1, 1, 0, 1), (2, 256, 3, -1, 2, 512, 1),
+                    (2, 512, 2, 4, 0, 128, 1), (2, 32, 1, 3, 2, 512, 1), (2, 8, 1, 1, 0, 256, 1), (1, 128, 0, 0, 0, 0, 0),
+                    (2, 0, 0, 0, 0, 0, 0), (2, 32, 0, 2, 0, 128, 2), (2, 64, 0, 1, 2, 512, 2), (2, 256, 0, 0, 1, 256, 2))
+        for path, cols, stages, tpc, tab, thr, mix in variants:
             B.set_tuning(0, path); B.set_tuning(1, cols); B.set_tuning(2, stages)
-            B.set_tuning(4, tpc); B.set_tuning(5, tab); B.set_tuning(6, thr); B.set_tuning(7, coop)
+            B.set_tuning(4, tpc); B.set_tuning(5, tab); B.set_tuning(6, thr); B.set_tuning(7, mix)
             x, m = x0.clone(), m0.clone()
             for k in range(3):
                 lib_rule(rule, topo, k, x, m, g, 0.9, 0.1)
             torch.cuda.synchronize()
             assert B.kernel_error() == 0
-            outs.append((x, m, path == 2 and coop in (0, 3)))
+            outs.append((x, m, path == 2 and mix in (0, 2)))
     finally:
         for knob in range(8):
             B.set_tuning(knob, 0)
