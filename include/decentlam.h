@@ -69,10 +69,17 @@ typedef enum dlm_topology_kind {
     DLM_TOPO_COMPLETE = 3,     /* w_ij = 1/n (Sec. 3: the fully connected case) */
     DLM_TOPO_CSR_MH = 4,       /* caller gives an undirected graph, weights by the Metropolis-Hastings
                                   rule cited under Assumption A.3: w_ij = 1/(1 + max(deg_i, deg_j)) */
-    DLM_TOPO_CSR_WEIGHTS = 5   /* caller gives W itself */
+    DLM_TOPO_CSR_WEIGHTS = 5,  /* caller gives W itself */
+    DLM_TOPO_SYM_EXP = 6,      /* symmetric exponential graph (App. G): every odd rank i is joined to the
+                                  even ranks (i + 2^t - 1) mod n, t = 1..floor(log2(n-1)); undirected,
+                                  Metropolis-Hastings weights; n even, n >= 4 */
+    DLM_TOPO_MESH = 7          /* logical mesh (App. G): r x c grid in row-major rank order, r the largest
+                                  divisor of n not above sqrt(n); direct neighbours, no wrap-around;
+                                  Metropolis-Hastings weights; n >= 2 */
 } dlm_topology_kind;
 
 #define DLM_MAX_NODES 2048
+#define DLM_MAX_PERIOD 4096
 
 /*
  * Build the tables for a topology on n nodes and upload them to the current device.
@@ -91,6 +98,18 @@ typedef enum dlm_topology_kind {
  */
 DLM_API int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
                    dlm_topology** out);
+
+/*
+ * Time-varying topology given slot by slot (App. G "Bipartite Random Match" and any other graph
+ * sequence: the caller draws the graphs, e.g. one random perfect matching per iteration, so that
+ * no random-number generator has to agree between programs).  Iteration k uses slot k mod period.
+ *   kind   : DLM_TOPO_CSR_MH or DLM_TOPO_CSR_WEIGHTS, with the per-slot requirements of topology_build.
+ *   rowptr : host int32[period * n + 1]: the slots' CSR row offsets concatenated; slot s owns rows
+ *            s*n .. (s+1)*n - 1 and its offsets index the shared col / val arrays.
+ * Errors: as topology_build, plus DLM_ERR_SHAPE for period < 1 or > DLM_MAX_PERIOD.
+ */
+DLM_API int topology_build_periodic(int kind, int n, int period, const int32_t* rowptr, const int32_t* col,
+                                    const float* val, dlm_topology** out);
 
 /* Number of distinct slots; iteration k uses slot k mod period (k = 0 is the first step). */
 DLM_API int topology_period(const dlm_topology* topo, int* period);

@@ -18,7 +18,7 @@ import numpy as np
 
 from . import build as _build
 
-RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, ADJ_MH = 0, 1, 2, 3, 4
+RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, ADJ_MH, SYM_EXP, MESH = 0, 1, 2, 3, 4, 5, 6
 
 _lib = None
 

@@ -52,7 +52,8 @@ double w32(int q) { return (double)(float)(1.0 / (double)q); }
 extern "C" {
 
 // Topology kinds understood by the oracle.
-enum { ORC_RING = 0, ORC_STATIC_EXP = 1, ORC_ONE_PEER_EXP = 2, ORC_COMPLETE = 3, ORC_ADJ_MH = 4 };
+enum { ORC_RING = 0, ORC_STATIC_EXP = 1, ORC_ONE_PEER_EXP = 2, ORC_COMPLETE = 3, ORC_ADJ_MH = 4,
+       ORC_SYM_EXP = 5, ORC_MESH = 6 };
 
 // Number of distinct weight matrices the topology cycles through (slot = k mod period).
 // One-peer exponential graph: one hop 2^t per iteration, t = 0 .. floor(log2(n-1)).
@@ -78,6 +79,13 @@ int orc_topology_period(int kind, int n) {
 //   ADJ_MH        Metropolis-Hastings rule (Assumption A.3 and App. G cite it without
 //                 printing it): w_ij = 1 / (1 + max(deg_i, deg_j)) on every edge, the
 //                 diagonal takes the remainder.
+//   SYM_EXP       symmetric exponential graph of App. G: every odd rank i is joined to the even
+//                 ranks (i + 2^t - 1) mod n, t = 1 .. floor(log2(n-1)) (the t = 0 term of the
+//                 printed list is i itself, and its last term is read with the "- 1" the others
+//                 carry); undirected; Metropolis-Hastings weights.  n even, n >= 4.
+//   MESH          logical mesh of App. G: nodes on an r x c grid (row-major ranks), r the largest
+//                 divisor of n not above sqrt(n), joined to their direct horizontal and
+//                 vertical neighbours, no wrap-around; Metropolis-Hastings weights.  n >= 2.
 int orc_topology_dense(int kind, int n, int slot, const uint8_t* adj, double* W) {
     if (n < 1 || !W) return -1;
     std::vector<int> q((size_t)n * n, 0);  // integer denominators, 0 = no edge
@@ -106,7 +114,34 @@ int orc_topology_dense(int kind, int n, int slot, const uint8_t* adj, double* W)
     case ORC_COMPLETE:
         for (int i = 0; i < n; ++i) for (int j = 0; j < n; ++j) if (i != j) Q(i, j) = n;
         break;
+    case ORC_SYM_EXP:
+    case ORC_MESH:
     case ORC_ADJ_MH: {
+        std::vector<uint8_t> built;
+        if (kind == ORC_SYM_EXP) {
+            if (n < 4 || n % 2) return -1;
+            built.assign((size_t)n * n, 0);
+            const int T = floor_log2(n - 1);
+            for (int i = 1; i < n; i += 2)
+                for (int t = 1; t <= T; ++t) {
+                    const int j = (int)(((int64_t)i + ((int64_t)1 << t) - 1) % n);
+                    built[(size_t)i * n + j] = built[(size_t)j * n + i] = 1;
+                }
+            adj = built.data();
+        } else if (kind == ORC_MESH) {
+            if (n < 2) return -1;
+            built.assign((size_t)n * n, 0);
+            int r = 1;
+            for (int c = 1; c * c <= n; ++c) if (n % c == 0) r = c;
+            const int cols = n / r;
+            for (int a = 0; a < r; ++a)
+                for (int b = 0; b < cols; ++b) {
+                    const int i = a * cols + b;
+                    if (b + 1 < cols) built[(size_t)i * n + i + 1] = built[(size_t)(i + 1) * n + i] = 1;
+                    if (a + 1 < r) built[(size_t)i * n + i + cols] = built[(size_t)(i + cols) * n + i] = 1;
+                }
+            adj = built.data();
+        }
         if (!adj) return -1;
         std::vector<int> deg(n, 0);
         for (int i = 0; i < n; ++i) {

@@ -11,7 +11,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdecentlam.so")
 
-RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, CSR_MH, CSR_WEIGHTS = range(6)
+RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, CSR_MH, CSR_WEIGHTS, SYM_EXP, MESH = range(8)
 G_F32, G_BF16 = 0, 1
 MAX_NODES = 2048
 
@@ -42,6 +42,7 @@ _flt = ctypes.c_float
 _lib.dlm_status_string.argtypes = [_int]
 _lib.dlm_status_string.restype = ctypes.c_char_p
 _lib.topology_build.argtypes = [_int, _int, _vp, _vp, _vp, ctypes.POINTER(_vp)]
+_lib.topology_build_periodic.argtypes = [_int, _int, _int, _vp, _vp, _vp, ctypes.POINTER(_vp)]
 _lib.topology_period.argtypes = [_vp, ctypes.POINTER(_int)]
 _lib.topology_nodes.argtypes = [_vp, ctypes.POINTER(_int)]
 for _name in ("topology_tables_host", "topology_tables_device"):
@@ -60,7 +61,7 @@ _lib.dlm_launch_count.restype = _i64
 _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
 _lib.dlm_set_tuning.argtypes = [_int, _int]
 
-EXPORTS = ["dlm_status_string", "topology_build", "topology_period", "topology_nodes", "topology_tables_host",
+EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
            "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "pmsgd_step",
            "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
@@ -138,6 +139,21 @@ def topology_build(kind, n, rowptr=None, col=None, val=None):
     keep_v, pv = ptr(val, np.float32)
     out = _vp()
     _check(_lib.topology_build(kind, n, pr, pc, pv, ctypes.byref(out)), "topology_build")
+    return Topology(out)
+
+
+def topology_build_periodic(kind, n, period, rowptr, col, val=None):
+    """Time-varying topology: concatenated CSR of `period` slots (rowptr has period * n + 1 entries)."""
+    import numpy as np
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    pv = None
+    if val is not None:
+        val = np.ascontiguousarray(val, dtype=np.float32)
+        pv = val.ctypes.data_as(_vp)
+    out = _vp()
+    _check(_lib.topology_build_periodic(kind, n, period, rowptr.ctypes.data_as(_vp), col.ctypes.data_as(_vp), pv,
+                                        ctypes.byref(out)), "topology_build_periodic")
     return Topology(out)
 
 

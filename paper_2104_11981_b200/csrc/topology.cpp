@@ -124,98 +124,149 @@ bool has_entry(const int32_t* rowptr, const int32_t* col, int i, int j) {
     return std::binary_search(col + rowptr[i], col + rowptr[i + 1], (int32_t)j);
 }
 
+// Metropolis-Hastings rows from symmetric adjacency lists (ascending, no self loops).
+void emit_mh_rows(int n, const std::vector<std::vector<int32_t>>& nbr, dlm_slot& s) {
+    for (int i = 0; i < n; ++i) {
+        std::vector<Edge> nb;
+        for (int32_t j : nbr[i])
+            nb.push_back({j, 1 + (int)std::max(nbr[i].size(), nbr[j].size())});
+        emit_row(i, nb, s);
+    }
+}
+
+// Fill one slot's host tables.  For the CSR kinds rowptr/col/val describe this slot only
+// (rowptr[0] == 0).
+int fill_slot(int kind, int n, int slot, const int32_t* rowptr, const int32_t* col, const float* val, dlm_slot& s) {
+    int rc = DLM_OK;
+    s.rowptr.push_back(0);
+    switch (kind) {
+    case DLM_TOPO_RING:
+        for (int i = 0; i < n; ++i)
+            emit_row(i, unique_neighbours(i, {(int32_t)((i + 1) % n), (int32_t)((i + n - 1) % n)}, 3), s);
+        break;
+    case DLM_TOPO_STATIC_EXP: {
+        int L = hops_of(n);
+        for (int i = 0; i < n; ++i) {
+            std::vector<int32_t> js;
+            for (int h = 0; h < L; ++h) js.push_back((int32_t)(((int64_t)i + (int64_t(1) << h)) % n));
+            emit_row(i, unique_neighbours(i, js, L + 1), s);
+        }
+        break;
+    }
+    case DLM_TOPO_ONE_PEER_EXP:
+        for (int i = 0; i < n; ++i)
+            emit_row(i, unique_neighbours(i, {(int32_t)(((int64_t)i + (int64_t(1) << slot)) % n)}, 2), s);
+        break;
+    case DLM_TOPO_COMPLETE:
+        for (int i = 0; i < n; ++i) {
+            std::vector<Edge> nb;
+            for (int j = 0; j < n; ++j)
+                if (j != i) nb.push_back({(int32_t)j, n});
+            emit_row(i, nb, s);
+        }
+        break;
+    case DLM_TOPO_SYM_EXP: {
+        // odd rank i <-> even ranks (i + 2^t - 1) mod n, t = 1 .. floor(log2(n-1)); undirected
+        std::vector<std::vector<int32_t>> nbr(n);
+        const int T = hops_of(n) - 1;
+        for (int i = 1; i < n; i += 2)
+            for (int h = 1; h <= T; ++h) {
+                const int32_t j = (int32_t)(((int64_t)i + (int64_t(1) << h) - 1) % n);
+                nbr[i].push_back(j);
+                nbr[j].push_back(i);
+            }
+        for (auto& v : nbr) { std::sort(v.begin(), v.end()); v.erase(std::unique(v.begin(), v.end()), v.end()); }
+        emit_mh_rows(n, nbr, s);
+        break;
+    }
+    case DLM_TOPO_MESH: {
+        // r x c grid, r the largest divisor of n not above sqrt(n); direct neighbours, no wrap-around
+        int r = 1;
+        for (int c = 1; c * c <= n; ++c) if (n % c == 0) r = c;
+        const int cols = n / r;
+        std::vector<std::vector<int32_t>> nbr(n);
+        for (int i = 0; i < n; ++i) {
+            const int a = i / cols, b = i % cols;
+            if (a > 0) nbr[i].push_back(i - cols);
+            if (b > 0) nbr[i].push_back(i - 1);
+            if (b + 1 < cols) nbr[i].push_back(i + 1);
+            if (a + 1 < r) nbr[i].push_back(i + cols);
+        }
+        emit_mh_rows(n, nbr, s);
+        break;
+    }
+    case DLM_TOPO_CSR_MH: {
+        if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
+        for (int i = 0; i < n && rc == DLM_OK; ++i)
+            for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p)
+                if (col[p] == i || !has_entry(rowptr, col, col[p], i)) { rc = DLM_ERR_TOPOLOGY; break; }
+        if (rc != DLM_OK) break;
+        for (int i = 0; i < n; ++i) {
+            int deg_i = rowptr[i + 1] - rowptr[i];
+            std::vector<Edge> nb;
+            for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                int j = col[p], deg_j = rowptr[j + 1] - rowptr[j];
+                nb.push_back({(int32_t)j, 1 + std::max(deg_i, deg_j)});
+            }
+            emit_row(i, nb, s);
+        }
+        break;
+    }
+    case DLM_TOPO_CSR_WEIGHTS: {
+        if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
+        std::vector<double> colsum(n, 0.0);
+        for (int i = 0; i < n && rc == DLM_OK; ++i) {
+            double rowsum = 0.0;
+            if (!has_entry(rowptr, col, i, i)) { rc = DLM_ERR_TOPOLOGY; break; }
+            for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                if (!(val[p] > 0.0f) || !std::isfinite(val[p])) { rc = DLM_ERR_TOPOLOGY; break; }
+                rowsum += (double)val[p];
+                colsum[col[p]] += (double)val[p];
+            }
+            if (rc == DLM_OK && std::fabs(rowsum - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
+        }
+        for (int j = 0; j < n && rc == DLM_OK; ++j)
+            if (std::fabs(colsum[j] - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
+        if (rc != DLM_OK) break;
+        s.rowptr.assign(rowptr, rowptr + n + 1);
+        s.col.assign(col, col + rowptr[n]);
+        s.val.assign(val, val + rowptr[n]);
+        for (int i = 0; i < n; ++i) s.max_degree = std::max(s.max_degree, rowptr[i + 1] - rowptr[i]);
+        break;
+    }
+    }
+    return rc;
+}
+
 }  // namespace
 
 extern "C" {
 
-int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
-                   dlm_topology** out) {
-    if (!out) return DLM_ERR_NULL;
-    *out = nullptr;
-    if (kind < DLM_TOPO_RING || kind > DLM_TOPO_CSR_WEIGHTS) return DLM_ERR_KIND;
-    if (n < 1) return DLM_ERR_SHAPE;
-    if (n > DLM_MAX_NODES) return DLM_ERR_UNSUPPORTED;
-    if (kind == DLM_TOPO_RING && n < 3) return DLM_ERR_SHAPE;
-    if ((kind == DLM_TOPO_STATIC_EXP || kind == DLM_TOPO_ONE_PEER_EXP) && n < 2) return DLM_ERR_SHAPE;
-    if (kind == DLM_TOPO_CSR_MH && (!rowptr || (!col && rowptr[n] > 0))) return DLM_ERR_NULL;
-    if (kind == DLM_TOPO_CSR_WEIGHTS && (!rowptr || !col || !val)) return DLM_ERR_NULL;
-
+static int build_common(int kind, int n, int period, const int32_t* rowptr, const int32_t* col, const float* val,
+                        dlm_topology** out) {
     dlm_topology* t = new (std::nothrow) dlm_topology;
     if (!t) return DLM_ERR_CUDA;
     t->n = n;
     t->kind = kind;
-    int period = (kind == DLM_TOPO_ONE_PEER_EXP) ? hops_of(n) : 1;
     t->slots.resize(period);
     int rc = DLM_OK;
-
+    const bool csr = kind == DLM_TOPO_CSR_MH || kind == DLM_TOPO_CSR_WEIGHTS;
     for (int slot = 0; slot < period && rc == DLM_OK; ++slot) {
-        dlm_slot& s = t->slots[slot];
-        s.rowptr.push_back(0);
-        switch (kind) {
-        case DLM_TOPO_RING:
-            for (int i = 0; i < n; ++i)
-                emit_row(i, unique_neighbours(i, {(int32_t)((i + 1) % n), (int32_t)((i + n - 1) % n)}, 3), s);
-            break;
-        case DLM_TOPO_STATIC_EXP: {
-            int L = hops_of(n);
-            for (int i = 0; i < n; ++i) {
-                std::vector<int32_t> js;
-                for (int h = 0; h < L; ++h) js.push_back((int32_t)(((int64_t)i + (int64_t(1) << h)) % n));
-                emit_row(i, unique_neighbours(i, js, L + 1), s);
+        if (csr) {
+            // slot s owns rows s*n .. (s+1)*n of the concatenated CSR; rebase it to start at 0
+            const int32_t* rp = rowptr + (size_t)slot * n;
+            const int32_t base = rp[0];
+            bool ok = base >= 0;
+            std::vector<int32_t> local(n + 1);
+            for (int i = 0; i <= n; ++i) {
+                local[i] = rp[i] - base;
+                if (rp[i] < base) ok = false;
             }
-            break;
-        }
-        case DLM_TOPO_ONE_PEER_EXP:
-            for (int i = 0; i < n; ++i)
-                emit_row(i, unique_neighbours(i, {(int32_t)(((int64_t)i + (int64_t(1) << slot)) % n)}, 2), s);
-            break;
-        case DLM_TOPO_COMPLETE:
-            for (int i = 0; i < n; ++i) {
-                std::vector<Edge> nb;
-                for (int j = 0; j < n; ++j)
-                    if (j != i) nb.push_back({(int32_t)j, n});
-                emit_row(i, nb, s);
-            }
-            break;
-        case DLM_TOPO_CSR_MH: {
-            if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
-            for (int i = 0; i < n && rc == DLM_OK; ++i)
-                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p)
-                    if (col[p] == i || !has_entry(rowptr, col, col[p], i)) { rc = DLM_ERR_TOPOLOGY; break; }
-            if (rc != DLM_OK) break;
-            for (int i = 0; i < n; ++i) {
-                int deg_i = rowptr[i + 1] - rowptr[i];
-                std::vector<Edge> nb;
-                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
-                    int j = col[p], deg_j = rowptr[j + 1] - rowptr[j];
-                    nb.push_back({(int32_t)j, 1 + std::max(deg_i, deg_j)});
-                }
-                emit_row(i, nb, s);
-            }
-            break;
-        }
-        case DLM_TOPO_CSR_WEIGHTS: {
-            if (!pattern_ok(n, rowptr, col)) { rc = DLM_ERR_TOPOLOGY; break; }
-            std::vector<double> colsum(n, 0.0);
-            for (int i = 0; i < n && rc == DLM_OK; ++i) {
-                double rowsum = 0.0;
-                if (!has_entry(rowptr, col, i, i)) { rc = DLM_ERR_TOPOLOGY; break; }
-                for (int32_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
-                    if (!(val[p] > 0.0f) || !std::isfinite(val[p])) { rc = DLM_ERR_TOPOLOGY; break; }
-                    rowsum += (double)val[p];
-                    colsum[col[p]] += (double)val[p];
-                }
-                if (rc == DLM_OK && std::fabs(rowsum - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
-            }
-            for (int j = 0; j < n && rc == DLM_OK; ++j)
-                if (std::fabs(colsum[j] - 1.0) > 1e-6) rc = DLM_ERR_TOPOLOGY;
-            if (rc != DLM_OK) break;
-            s.rowptr.assign(rowptr, rowptr + n + 1);
-            s.col.assign(col, col + rowptr[n]);
-            s.val.assign(val, val + rowptr[n]);
-            for (int i = 0; i < n; ++i) s.max_degree = std::max(s.max_degree, rowptr[i + 1] - rowptr[i]);
-            break;
-        }
+            if (!ok) { rc = DLM_ERR_TOPOLOGY; break; }
+            rc = fill_slot(kind, n, slot, local.data(), col ? col + base : nullptr, val ? val + base : nullptr,
+                           t->slots[slot]);
+        } else {
+            rc = fill_slot(kind, n, slot, nullptr, nullptr, nullptr, t->slots[slot]);
         }
     }
     for (int slot = 0; slot < period && rc == DLM_OK; ++slot) make_order(t->slots[slot]);
@@ -232,6 +283,35 @@ int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, c
     }
     *out = t;
     return DLM_OK;
+}
+
+int topology_build(int kind, int n, const int32_t* rowptr, const int32_t* col, const float* val,
+                   dlm_topology** out) {
+    if (!out) return DLM_ERR_NULL;
+    *out = nullptr;
+    if (kind < DLM_TOPO_RING || kind > DLM_TOPO_MESH) return DLM_ERR_KIND;
+    if (n < 1) return DLM_ERR_SHAPE;
+    if (n > DLM_MAX_NODES) return DLM_ERR_UNSUPPORTED;
+    if (kind == DLM_TOPO_RING && n < 3) return DLM_ERR_SHAPE;
+    if ((kind == DLM_TOPO_STATIC_EXP || kind == DLM_TOPO_ONE_PEER_EXP || kind == DLM_TOPO_MESH) && n < 2)
+        return DLM_ERR_SHAPE;
+    if (kind == DLM_TOPO_SYM_EXP && (n < 4 || n % 2)) return DLM_ERR_SHAPE;
+    if (kind == DLM_TOPO_CSR_MH && (!rowptr || (!col && rowptr[n] > 0))) return DLM_ERR_NULL;
+    if (kind == DLM_TOPO_CSR_WEIGHTS && (!rowptr || !col || !val)) return DLM_ERR_NULL;
+    const int period = (kind == DLM_TOPO_ONE_PEER_EXP) ? hops_of(n) : 1;
+    return build_common(kind, n, period, rowptr, col, val, out);
+}
+
+int topology_build_periodic(int kind, int n, int period, const int32_t* rowptr, const int32_t* col,
+                            const float* val, dlm_topology** out) {
+    if (!out) return DLM_ERR_NULL;
+    *out = nullptr;
+    if (kind != DLM_TOPO_CSR_MH && kind != DLM_TOPO_CSR_WEIGHTS) return DLM_ERR_KIND;
+    if (n < 1 || period < 1 || period > DLM_MAX_PERIOD) return DLM_ERR_SHAPE;
+    if (n > DLM_MAX_NODES) return DLM_ERR_UNSUPPORTED;
+    if (!rowptr || (!col && rowptr[(size_t)period * n] > rowptr[0])) return DLM_ERR_NULL;
+    if (kind == DLM_TOPO_CSR_WEIGHTS && (!col || !val)) return DLM_ERR_NULL;
+    return build_common(kind, n, period, rowptr, col, val, out);
 }
 
 int topology_period(const dlm_topology* topo, int* period) {

@@ -115,6 +115,33 @@ def adjacency_to_lists(adj):
     return rowptr, (np.concatenate(cols) if cols else np.zeros(0, np.int32)).astype(np.int32)
 
 
+def bipartite_matchings(n, period, seed):
+    """`period` random perfect matchings of n nodes (n even), one per iteration, as App. G's
+    "bipartite random match": the nodes are split at random into two halves and paired.
+    Returns a list of symmetric 0/1 adjacency matrices [n, n] (uint8), each of degree one."""
+    assert n % 2 == 0
+    rng = np.random.Generator(np.random.Philox(seed))
+    out = []
+    for _ in range(period):
+        perm = rng.permutation(n)
+        adj = np.zeros((n, n), dtype=np.uint8)
+        for a, b in zip(perm[: n // 2], perm[n // 2:]):
+            adj[a, b] = adj[b, a] = 1
+        out.append(adj)
+    return out
+
+
+def concat_adjacency_lists(adjs):
+    """Concatenated CSR (rowptr int32[period*n+1], col) of several adjacency matrices of equal size."""
+    rowptrs, cols, base = [np.zeros(1, np.int32)], [], 0
+    for adj in adjs:
+        rp, c = adjacency_to_lists(adj)
+        rowptrs.append(rp[1:] + base)
+        cols.append(c)
+        base += len(c)
+    return np.concatenate(rowptrs).astype(np.int32), np.concatenate(cols).astype(np.int32)
+
+
 def lsq_problem_np(n, p, q, seed, hetero=0.5, noise_std=0.01):
     """Least-squares data of the linear-regression experiment (App. G), heterogeneous variant:
     A_i ~ N(0,1) [p, q];  b_i = A_i (x_o + hetero * u_i) + N(0, noise_std), x_o, u_i ~ N(0,1).

@@ -8,15 +8,20 @@ import oracle
 from paper_2104_11981_b200 import inputs
 
 ORACLE_KIND = {"ring": oracle.RING, "static_exp": oracle.STATIC_EXP, "one_peer_exp": oracle.ONE_PEER_EXP,
-               "complete": oracle.COMPLETE, "er_mh": oracle.ADJ_MH}
+               "complete": oracle.COMPLETE, "er_mh": oracle.ADJ_MH, "sym_exp": oracle.SYM_EXP, "mesh": oracle.MESH}
 THREADS = max(1, os.cpu_count() or 1)
 
 
-def build_both(topology, n, graph_seed=None, er_p=0.05):
+def build_both(topology, n, graph_seed=None, er_p=0.05, period=8):
     """Returns (library Topology, [dense oracle W per slot])."""
     from paper_2104_11981_b200 import binding as B
+    if topology == "bipartite_match":
+        adjs = inputs.bipartite_matchings(n, period, graph_seed)
+        rowptr, col = inputs.concat_adjacency_lists(adjs)
+        topo = B.topology_build_periodic(B.CSR_MH, n, period, rowptr, col)
+        return topo, [oracle.topology_dense(oracle.ADJ_MH, n, 0, a) for a in adjs]
     lib_kind = {"ring": B.RING, "static_exp": B.STATIC_EXP, "one_peer_exp": B.ONE_PEER_EXP,
-                "complete": B.COMPLETE, "er_mh": B.CSR_MH}[topology]
+                "complete": B.COMPLETE, "er_mh": B.CSR_MH, "sym_exp": B.SYM_EXP, "mesh": B.MESH}[topology]
     adj = None
     if topology == "er_mh":
         adj, _ = inputs.er_adjacency(n, er_p, graph_seed)

@@ -77,6 +77,52 @@ def test_mh_tables_bit_exact(n, p, seed):
     _check_tables(B.topology_build(B.CSR_MH, n, rowptr, col), oracle.ADJ_MH, n, adj)
 
 
+@pytest.mark.parametrize("n", [4, 8, 12, 16, 64, 100])
+def test_symmetric_exponential_tables_bit_exact(n):
+    _check_tables(B.topology_build(B.SYM_EXP, n), oracle.SYM_EXP, n)
+
+
+@pytest.mark.parametrize("n", [2, 7, 8, 12, 16, 64])
+def test_mesh_tables_bit_exact(n):
+    _check_tables(B.topology_build(B.MESH, n), oracle.MESH, n)
+
+
+def test_periodic_tables_bit_exact_and_validation():
+    """Bipartite random match: one matching per slot, handed to both sides as adjacency."""
+    n, period = 16, 6
+    adjs = inputs.bipartite_matchings(n, period, 21)
+    rowptr, col = inputs.concat_adjacency_lists(adjs)
+    topo = B.topology_build_periodic(B.CSR_MH, n, period, rowptr, col)
+    assert topo.period == period and topo.n == n
+    for s in range(period):
+        rp, c, v = topo.tables_host(s)
+        Wo = oracle.topology_dense(oracle.ADJ_MH, n, 0, adjs[s])
+        assert np.array_equal(_dense_from_csr(n, rp, c, v).view(np.uint32), Wo.astype(np.float32).view(np.uint32))
+    # explicit weights, two slots (ring, then identity)
+    W = oracle.topology_dense(oracle.RING, 4).astype(np.float32)
+    rp = [0]; cc = []; vv = []
+    for i in range(4):
+        js = sorted({(i - 1) % 4, i, (i + 1) % 4}); cc += js; vv += [W[i, j] for j in js]; rp.append(len(cc))
+    for i in range(4):
+        cc.append(i); vv.append(1.0); rp.append(len(cc))
+    t2 = B.topology_build_periodic(B.CSR_WEIGHTS, 4, 2, np.array(rp), np.array(cc), np.array(vv, np.float32))
+    assert t2.period == 2 and np.array_equal(t2.tables_host(1)[1], np.arange(4)) and np.all(t2.tables_host(1)[2] == 1.0)
+
+    def expect(status, *args):
+        with pytest.raises(B.DecentlamError) as e:
+            B.topology_build_periodic(*args)
+        assert e.value.status == status
+
+    expect(-6, B.RING, n, period, rowptr, col)
+    expect(-2, B.CSR_MH, n, 0, rowptr, col)
+    expect(-2, B.CSR_MH, n, 5000, rowptr, col)
+    bad = rowptr.copy(); bad[n + 3] = bad[n + 2] - 1       # offsets running backwards inside slot 1
+    expect(-7, B.CSR_MH, n, period, bad, col)
+    badc = col.copy(); badc[0] = (badc[0] + 1) % n           # breaks the symmetry of slot 0
+    expect(-7, B.CSR_MH, n, period, rowptr, badc)
+    assert B.raw().topology_build_periodic(B.CSR_MH, n, period, None, None, None, ctypes.byref(ctypes.c_void_p())) == -1
+
+
 def test_csr_weights_roundtrip_and_validation():
     W = oracle.topology_dense(oracle.RING, 6).astype(np.float32)
     rowptr = np.arange(0, 19, 3, dtype=np.int32)
@@ -107,6 +153,9 @@ def test_csr_weights_roundtrip_and_validation():
     expect(-6, 17, 4)
     expect(-2, B.RING, 2)
     expect(-2, B.STATIC_EXP, 1)
+    expect(-2, B.SYM_EXP, 7)
+    expect(-2, B.SYM_EXP, 2)
+    expect(-2, B.MESH, 1)
     expect(-8, B.COMPLETE, B.MAX_NODES + 1)
     expect(-1, B.CSR_WEIGHTS, 4)
     lib = B.raw()

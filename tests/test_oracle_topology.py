@@ -16,6 +16,12 @@ def _all_cases():
             cases.append((oracle.ONE_PEER_EXP, n, s, None))
     for n in (1, 2, 7):
         cases.append((oracle.COMPLETE, n, 0, None))
+    for n in (4, 8, 12, 16, 64, 100):
+        cases.append((oracle.SYM_EXP, n, 0, None))
+    for n in (2, 7, 8, 12, 16, 64):
+        cases.append((oracle.MESH, n, 0, None))
+    for adj in inputs.bipartite_matchings(16, 3, 11):
+        cases.append((oracle.ADJ_MH, 16, 0, adj))
     for n, p, seed in ((8, 0.4, 1), (40, 0.2, 2), (256, 0.05, 3)):
         adj, _ = inputs.er_adjacency(n, p, seed)
         cases.append((oracle.ADJ_MH, n, 0, adj))
@@ -139,3 +145,50 @@ def test_spectral_gap_of_symmetric_graphs():
         lam = np.sort(np.linalg.eigvalsh(W))[::-1]
         assert abs(lam[0] - 1.0) < 1e-6
         assert max(abs(lam[1]), abs(lam[-1])) < 1.0 - 1e-3
+
+
+def test_symmetric_exponential_graph_neighbours():
+    """App. G: odd rank i talks to the even ranks i + 2^t - 1.  n = 8: floor(log2 7) = 2, so odd i is
+    joined to i + 1 and i + 3 (mod 8); every node then has exactly two peers and weight 1/3."""
+    n = 8
+    W = oracle.topology_dense(oracle.SYM_EXP, n)
+    assert np.array_equal(W, W.T)
+    for i in range(1, n, 2):
+        assert set(np.nonzero(W[i])[0]) == {i, (i + 1) % n, (i + 3) % n}
+    for i in range(0, n, 2):
+        assert set(np.nonzero(W[i])[0]) == {i, (i - 1) % n, (i - 3) % n}
+    assert np.all(W[W > 0] == np.float64(np.float32(1.0 / 3.0)))
+    # bipartite between odd and even ranks, and connected (spectral gap)
+    for n in (8, 16, 64):
+        W = oracle.topology_dense(oracle.SYM_EXP, n)
+        assert not W[0::2, 0::2][~np.eye(n // 2, dtype=bool)].any() and not W[1::2, 1::2][~np.eye(n // 2, dtype=bool)].any()
+        assert np.count_nonzero(W[1]) == 1 + int(np.floor(np.log2(n - 1)))
+        lam = np.sort(np.linalg.eigvalsh(W))[::-1]
+        assert abs(lam[0] - 1) < 1e-6 and max(abs(lam[1]), abs(lam[-1])) < 1 - 1e-3
+    with pytest.raises(ValueError):
+        oracle.topology_dense(oracle.SYM_EXP, 7)
+
+
+def test_mesh_neighbours():
+    """App. G: logical mesh, direct neighbours.  n = 8 is laid out 2 x 4: corners have 2 peers, the
+    others 3; n = 16 is 4 x 4 with 2 / 3 / 4 peers; Metropolis-Hastings weights."""
+    W = oracle.topology_dense(oracle.MESH, 8)
+    assert np.array_equal(W, W.T)
+    assert set(np.nonzero(W[0])[0]) == {0, 1, 4} and set(np.nonzero(W[5])[0]) == {1, 4, 5, 6}
+    assert W[0, 1] == 0.25 and W[0, 4] == np.float64(np.float32(1.0 / 3.0))      # 1/(1+max(2,3)), 1/(1+max(2,2))
+    W = oracle.topology_dense(oracle.MESH, 16)
+    deg = (W > 0).sum(1) - 1
+    assert sorted(deg) == [2] * 4 + [3] * 8 + [4] * 4
+    assert set(np.nonzero(W[5])[0]) == {1, 4, 5, 6, 9}
+    W7 = oracle.topology_dense(oracle.MESH, 7)                                    # prime: a 1 x 7 path
+    assert set(np.nonzero(W7[3])[0]) == {2, 3, 4} and set(np.nonzero(W7[0])[0]) == {0, 1}
+
+
+def test_bipartite_random_match_is_pairwise_averaging():
+    """App. G: the nodes are split into two halves and paired, each pair averages.  With
+    Metropolis-Hastings weights a degree-one graph gives 1/2, 1/2, so W is a symmetric projection."""
+    for adj in inputs.bipartite_matchings(12, 4, 5):
+        assert (adj.sum(1) == 1).all() and np.array_equal(adj, adj.T)
+        W = oracle.topology_dense(oracle.ADJ_MH, 12, 0, adj)
+        assert np.array_equal(W, W.T) and np.all(W[W > 0] == 0.5)
+        np.testing.assert_allclose(W @ W, W, atol=0)
