@@ -300,12 +300,15 @@ def run_ours(args):
 
     extra = {}
     if not args.no_extra and world == 1:
-        for name, fn in (("dmsgd", lambda k: B.dmsgd_step(topo, k, x, m, g, w.beta, w.gamma)),
-                         ("pmsgd", lambda k: B.pmsgd_step(x, m, g, w.beta, w.gamma))):
+        dsgd_bytes = 8 + g.element_size()     # no momentum: x, g read, x written
+        for name, fn, bpn in (("dmsgd", lambda k: B.dmsgd_step(topo, k, x, m, g, w.beta, w.gamma), bytes_per_np),
+                              ("pmsgd", lambda k: B.pmsgd_step(x, m, g, w.beta, w.gamma), bytes_per_np),
+                              ("dsgd_atc", lambda k: B.dsgd_step(topo, k, x, g, w.gamma, B.DSGD_ATC), dsgd_bytes),
+                              ("dsgd_awc", lambda k: B.dsgd_step(topo, k, x, g, w.gamma, B.DSGD_AWC), dsgd_bytes)):
             steps_x = max(10, args.steps // 2)
             s, _ = time_steps(fn, reset, steps_x, 3, torch, stream)
             extra[name] = {"ms_per_step": s / steps_x * 1e3, "value": n * d * steps_x / s,
-                           "gbs": bytes_per_np * n * d * steps_x / s / 1e9}
+                           "gbs": bpn * n * d * steps_x / s / 1e9}
 
     e2e = None
     if not args.no_e2e:

@@ -169,6 +169,20 @@ DLM_API int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, in
                float beta, float gamma, void* cuda_stream);
 
 /*
+ * Decentralized SGD without momentum (Sec. 3, Eqs. dsgd-1, dsgd-2; Remark in Sec. 5).  x is updated in
+ * place, there is no m; traffic is x and g read once, x written once (12 bytes per node-parameter).
+ *   variant DLM_DSGD_ATC  adapt-then-combine, the DSGD of Sec. 3:  y_i = x_i - gamma g_i ;
+ *                         x_i <- y_i + sum_{j != i} w_ij (y_j - y_i)            (= W (x - gamma g))
+ *                         (bitwise the x that dmsgd_step gives with beta = 0)
+ *   variant DLM_DSGD_AWC  adapt-with-combine of the Remark in Sec. 5:
+ *                         x_i <- x_i + sum_{j != i} w_ij (x_j - x_i) - gamma g_i  (= W x - gamma g)
+ * Other arguments and errors as for decentlam_step (no beta; DLM_ERR_KIND for an unknown variant).
+ */
+enum { DLM_DSGD_ATC = 0, DLM_DSGD_AWC = 1 };
+DLM_API int dsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, const void* g,
+                      int g_dtype, int64_t ldg, float gamma, int variant, void* cuda_stream);
+
+/*
  * Parallel momentum SGD on the globally averaged gradient (Sec. 1, Sec. 7 "PmSGD"):
  *   gbar = (1/n) sum_i g_i ;  m_i <- beta m_i + gbar ;  x_i <- x_i - gamma m_i(new)
  * No topology: the global average plays the role of W = (1/n) 1 1^T.

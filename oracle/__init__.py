@@ -42,6 +42,8 @@ def _L():
             f.restype = None
         _lib.orc_decentlam_step_pernode.argtypes = [ci, i64, dp, dp, dp, dp, cd, cd, dp, dp]
         _lib.orc_decentlam_step_pernode.restype = None
+        _lib.orc_dsgd_step.argtypes = [ci, i64, dp, dp, dp, cd, ci, dp, ci]
+        _lib.orc_dsgd_step.restype = None
         _lib.orc_pmsgd_step.argtypes = [ci, i64, dp, dp, dp, cd, cd, dp, dp, ci]
         _lib.orc_pmsgd_step.restype = None
         for name in ("orc_decentlam_two_term", "orc_dmsgd_two_term"):
@@ -97,6 +99,15 @@ def decentlam_step(W, x, m, g, beta, gamma, threads=1):
 def dmsgd_step(W, x, m, g, beta, gamma, threads=1):
     """One DmSGD iteration (Algorithm 1). Returns (x', m')."""
     return _step(_L().orc_dmsgd_step, W, x, m, g, beta, gamma, threads)
+
+
+def dsgd_step(W, x, g, gamma, variant=0, threads=1):
+    """DSGD without momentum: variant 0 = W(x - gamma g) (Sec. 3), variant 1 = W x - gamma g (Remark, Sec. 5)."""
+    W, x, g = _d(W), _d(x), _d(g)
+    n, d = x.shape
+    out = np.empty_like(x)
+    _L().orc_dsgd_step(n, d, _p(W), _p(x), _p(g), float(gamma), int(variant), _p(out), int(threads))
+    return out
 
 
 def decentlam_step_pernode(W, x, m, g, beta, gamma):

@@ -238,6 +238,28 @@ void orc_dmsgd_step(int n, int64_t d, const double* W, const double* x, const do
     });
 }
 
+// Decentralized SGD without momentum.
+//   variant 0, adapt-then-combine (Sec. 3, Eqs. dsgd-1, dsgd-2):  y = x - gamma g ;  x' = W y
+//   variant 1, adapt-with-combine (Remark in Sec. 5):             x' = W x - gamma g
+// W is applied with exact unit row sums: (W y)_i = y_i + sum_{j != i} w_ij (y_j - y_i).
+void orc_dsgd_step(int n, int64_t d, const double* W, const double* x, const double* g, double gamma, int variant,
+                   double* x_out, int threads) {
+    for_column_ranges(d, threads, [&](int64_t c0, int64_t c1) {
+        std::vector<double> y(n);
+        for (int64_t c = c0; c < c1; ++c) {
+            for (int i = 0; i < n; ++i)
+                y[i] = variant == 0 ? x[(size_t)i * d + c] - gamma * g[(size_t)i * d + c] : x[(size_t)i * d + c];
+            for (int i = 0; i < n; ++i) {
+                double acc = 0.0;
+                for (int j = 0; j < n; ++j) if (j != i) acc += W[(size_t)i * n + j] * (y[j] - y[i]);
+                double v = y[i] + acc;
+                if (variant == 1) v -= gamma * g[(size_t)i * d + c];
+                x_out[(size_t)i * d + c] = v;
+            }
+        }
+    });
+}
+
 // Parallel momentum SGD (Sec. 1 and Sec. 7: every node applies momentum SGD to the
 // globally averaged gradient):  gbar = (1/n) sum_i g_i ;  m'_i = beta m_i + gbar ;
 // x'_i = x_i - gamma m'_i.

@@ -13,6 +13,7 @@ LIB_PATH = os.path.join(_HERE, "libdecentlam.so")
 
 RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, CSR_MH, CSR_WEIGHTS, SYM_EXP, MESH = range(8)
 G_F32, G_BF16 = 0, 1
+DSGD_ATC, DSGD_AWC = 0, 1
 MAX_NODES = 2048
 
 STATUS = {0: "DLM_OK", -1: "DLM_ERR_NULL", -2: "DLM_ERR_SHAPE", -3: "DLM_ERR_ALIGN", -4: "DLM_ERR_ALIAS",
@@ -51,6 +52,7 @@ for _name in ("topology_tables_host", "topology_tables_device"):
 _lib.topology_destroy.argtypes = [_vp]
 for _name in ("decentlam_step", "dmsgd_step"):
     getattr(_lib, _name).argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
+_lib.dsgd_step.argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _int, _i64, _flt, _int, _vp]
 _lib.pmsgd_step.argtypes = [_int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
 _lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
 _lib.lsq_grad_workspace_bytes.restype = _i64
@@ -62,7 +64,7 @@ _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
 _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
-           "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "pmsgd_step",
+           "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "dsgd_step", "pmsgd_step",
            "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
@@ -189,6 +191,18 @@ def dmsgd_step(topo, k, x, m, g, beta, gamma, stream=None):
     n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
     _check(_lib.dmsgd_step(topo.handle, k, n, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)),
            "dmsgd_step")
+
+
+def dsgd_step(topo, k, x, g, gamma, variant=DSGD_ATC, stream=None):
+    import torch
+    assert x.is_cuda and g.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and g.shape == x.shape
+    assert x.stride(1) == 1 and g.stride(1) == 1
+    gd = G_F32 if g.dtype == torch.float32 else G_BF16 if g.dtype == torch.bfloat16 else None
+    if gd is None:
+        raise TypeError("g must be float32 or bfloat16")
+    n, d = x.shape
+    _check(_lib.dsgd_step(topo.handle, k, n, d, x.stride(0), _vp(x.data_ptr()), _vp(g.data_ptr()), gd, g.stride(0),
+                          gamma, variant, _stream_ptr(stream)), "dsgd_step")
 
 
 def pmsgd_step(x, m, g, beta, gamma, stream=None):

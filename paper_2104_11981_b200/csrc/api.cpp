@@ -37,10 +37,24 @@ int check_state(int n, int64_t d, int64_t ld, const float* x, const float* m, co
     return DLM_OK;
 }
 
+int check_dsgd(int n, int64_t d, int64_t ld, const float* x, const void* g, int g_dtype, int64_t ldg, float gamma) {
+    if (!x || !g) return DLM_ERR_NULL;
+    if (g_dtype != DLM_G_F32 && g_dtype != DLM_G_BF16) return DLM_ERR_KIND;
+    if (n < 1 || d < 1 || ld < d || ldg < d) return DLM_ERR_SHAPE;
+    if (n > DLM_MAX_NODES) return DLM_ERR_UNSUPPORTED;
+    const size_t gsz = g_dtype == DLM_G_BF16 ? 2 : 4;
+    if ((uintptr_t)x % 4 || (uintptr_t)g % gsz) return DLM_ERR_ALIGN;
+    if (!std::isfinite(gamma) || !(gamma > 0.0f)) return DLM_ERR_HYPER;
+    if (overlap(span(x, n, d, ld, 4), span(g, n, d, ldg, gsz))) return DLM_ERR_ALIAS;
+    return DLM_OK;
+}
+
 int topo_step(int rule, const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, float* m,
               const void* g, int g_dtype, int64_t ldg, float beta, float gamma, void* stream) {
     if (!topo) return DLM_ERR_NULL;
-    int rc = check_state(n, d, ld, x, m, g, g_dtype, ldg, beta, gamma);
+    const bool has_m = rule == DLM_RULE_DECENTLAM || rule == DLM_RULE_DMSGD;
+    int rc = has_m ? check_state(n, d, ld, x, m, g, g_dtype, ldg, beta, gamma)
+                   : check_dsgd(n, d, ld, x, g, g_dtype, ldg, gamma);
     if (rc != DLM_OK) return rc;
     if (n != topo->n || k < 0) return DLM_ERR_SHAPE;
     const dlm_slot& s = topo->slots[(size_t)(k % (int64_t)topo->slots.size())];
@@ -99,6 +113,13 @@ int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_
 int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, float* m,
                const void* g, int g_dtype, int64_t ldg, float beta, float gamma, void* cuda_stream) {
     return topo_step(DLM_RULE_DMSGD, topo, k, n, d, ld, x, m, g, g_dtype, ldg, beta, gamma, cuda_stream);
+}
+
+int dsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, const void* g,
+              int g_dtype, int64_t ldg, float gamma, int variant, void* cuda_stream) {
+    if (variant != DLM_DSGD_ATC && variant != DLM_DSGD_AWC) return DLM_ERR_KIND;
+    return topo_step(variant == DLM_DSGD_ATC ? DLM_RULE_DSGD_ATC : DLM_RULE_DSGD_AWC, topo, k, n, d, ld, x, nullptr, g,
+                     g_dtype, ldg, 0.0f, gamma, cuda_stream);
 }
 
 int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype, int64_t ldg,

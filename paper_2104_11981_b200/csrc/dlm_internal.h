@@ -29,7 +29,7 @@ struct dlm_topology {
     std::vector<dlm_slot> slots;
 };
 
-enum dlm_rule { DLM_RULE_DECENTLAM = 0, DLM_RULE_DMSGD = 1 };
+enum dlm_rule { DLM_RULE_DECENTLAM = 0, DLM_RULE_DMSGD = 1, DLM_RULE_DSGD_ATC = 2, DLM_RULE_DSGD_AWC = 3 };
 
 // Arguments of one fused step over the columns [0, d) of row-major [n, ld] arrays.
 struct dlm_step_args {

@@ -195,6 +195,13 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
                 if (RULE == DLM_RULE_DECENTLAM) {
                     st_f32<VEC>(xs + (size_t)i * C + off, xi);
                     st_f32<VEC>(gs + (size_t)i * C + off, gi);
+                } else if (RULE == DLM_RULE_DSGD_ATC) {  // y = x - gamma g
+                    Pack<VEC> y;
+#pragma unroll
+                    for (int u = 0; u < VEC; ++u) y.v[u] = fmaf(-a.gamma, gi.v[u], xi.v[u]);
+                    st_f32<VEC>(xs + (size_t)i * C + off, y);
+                } else if (RULE == DLM_RULE_DSGD_AWC) {  // mix x itself, the gradient is applied after
+                    st_f32<VEC>(xs + (size_t)i * C + off, xi);
                 } else {
                     const Pack<VEC> mi = ld_f32<VEC>(a.m + (size_t)i * a.ld + c);
                     Pack<VEC> mn, y;
@@ -218,6 +225,11 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
                     st_f32<VEC>(a.m + (size_t)i * a.ld + c, mn);
                 } else {
                     dmsgd_item<VEC>(t, i, off, C, xs, xn);
+                    if (RULE == DLM_RULE_DSGD_AWC) {
+                        const Pack<VEC> gi = ld_g<VEC>(g + (size_t)i * a.ldg + c);
+#pragma unroll
+                        for (int u = 0; u < VEC; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
+                    }
                 }
                 st_f32<VEC>(a.x + (size_t)i * a.ld + c, xn);
             }
@@ -271,6 +283,7 @@ struct TmaGeom {
     int cv_shift;    // log2(box_cols / 4)
     int stages;
     uint32_t x_bytes, g_bytes, stage_bytes;  // per-stage tile sizes (128-byte multiples)
+    uint32_t m_off, g_off;                   // byte offsets of the m and g tiles inside a stage
     uint32_t tx_bytes;                       // bytes one stage's three copies deliver
     int tables_in_smem;
     long long num_tiles;
@@ -302,8 +315,9 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         mbar_expect_tx(bar, geo.tx_bytes);
         for (int b = 0; b < geo.boxes; ++b) {
             tma_load_2d(dst + b * sub_x, &tm_x, c0 + b * Cb, 0, bar);
-            tma_load_2d(dst + 2 * geo.x_bytes + b * sub_g, &tm_g, c0 + b * Cb, 0, bar);
-            tma_load_2d(dst + geo.x_bytes + b * sub_x, &tm_m, c0 + b * Cb, 0, bar);
+            tma_load_2d(dst + geo.g_off + b * sub_g, &tm_g, c0 + b * Cb, 0, bar);
+            if (RULE == DLM_RULE_DECENTLAM || RULE == DLM_RULE_DMSGD)  // the DSGD rules have no momentum
+                tma_load_2d(dst + geo.m_off + b * sub_x, &tm_m, c0 + b * Cb, 0, bar);
         }
     };
 
@@ -334,24 +348,30 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         unsigned char* st = base + (size_t)s * geo.stage_bytes;
         const long long tile_base = (first + it * gridDim.x) * C;
 
-        if (RULE == DLM_RULE_DMSGD) {
+        if (RULE == DLM_RULE_DMSGD || RULE == DLM_RULE_DSGD_ATC) {
             for (int b = 0; b < geo.boxes; ++b) {
                 float* xs = reinterpret_cast<float*>(st + b * sub_x);
-                const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes + b * sub_x);
-                const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes + b * sub_g);
+                const float* ms = reinterpret_cast<const float*>(st + geo.m_off + b * sub_x);
+                const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off + b * sub_g);
                 const long long c_base = tile_base + (long long)b * Cb;
                 for (int e = threadIdx.x; e < items; e += blockDim.x) {
                     const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;   // any order: purely local
                     const long long c = c_base + off;
                     if (c < a.d) {
                         const Pack<4> xi = ld_f32<4>(xs + i * Cb + off);
-                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
                         const Pack<4> gi = ld_g<4>(gs + i * Cb + off);
-                        Pack<4> mn, y;
+                        Pack<4> y;
+                        if (RULE == DLM_RULE_DMSGD) {
+                            const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
+                            Pack<4> mn;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], y.v[u]);
-                        st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                            for (int u = 0; u < 4; ++u)
+                                dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], y.v[u]);
+                            st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) y.v[u] = fmaf(-a.gamma, gi.v[u], xi.v[u]);
+                        }
                         st_f32<4>(xs + i * Cb + off, y);
                     }
                 }
@@ -360,8 +380,8 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         }
         for (int b = 0; b < geo.boxes; ++b) {
             const float* xs = reinterpret_cast<const float*>(st + b * sub_x);
-            const float* ms = reinterpret_cast<const float*>(st + geo.x_bytes + b * sub_x);
-            const GT* gs = reinterpret_cast<const GT*>(st + 2 * geo.x_bytes + b * sub_g);
+            const float* ms = reinterpret_cast<const float*>(st + geo.m_off + b * sub_x);
+            const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off + b * sub_g);
             const long long c_base = tile_base + (long long)b * Cb;
             for (int e = threadIdx.x; e < items; e += blockDim.x) {
                 const int i = t.order[e >> geo.cv_shift], off = (e & cv_mask) * 4;
@@ -375,6 +395,11 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
                         st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
                     } else {
                         dmsgd_item<4>(t, i, off, Cb, xs, xn);
+                        if (RULE == DLM_RULE_DSGD_AWC) {
+                            const Pack<4> gi = ld_g<4>(gs + i * Cb + off);
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
+                        }
                     }
                     st_f32<4>(a.x + (size_t)i * a.ld + c, xn);
                 }
@@ -670,10 +695,11 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     const int tables_in_smem = g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
     const size_t fixed = 128 + kMaxStages * 8 + 16 + (tables_in_smem ? tab : 0);
     const size_t budget = (size_t)dev.smem_optin;
+    constexpr bool HAS_M = RULE == DLM_RULE_DECENTLAM || RULE == DLM_RULE_DMSGD;
     auto stage_bytes_for = [&](int C, uint32_t& xb, uint32_t& gb) {
         xb = (uint32_t)(((size_t)a.n * C * 4 + 127) & ~(size_t)127);
         gb = (uint32_t)(((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127);
-        return (size_t)2 * xb + gb;
+        return (size_t)(HAS_M ? 2 : 1) * xb + gb;
     };
     // Defaults (measured on B200): about 16 KB per staged array with row segments of at least
     // 128 bytes, ONE stage per CTA and a grid of many short-lived CTAs, several resident per SM.
@@ -699,7 +725,8 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     const int box_cols = std::min(C, 256);
 
     CUtensorMap tm_x, tm_m, tm_g;
-    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, box_cols) || !make_map(&tm_m, a.m, false, a.n, a.d, a.ld, box_cols) ||
+    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, box_cols) ||
+        !make_map(&tm_m, HAS_M ? a.m : a.x, false, a.n, a.d, a.ld, box_cols) ||
         !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, box_cols))
         return DLM_ERR_UNSUPPORTED;
 
@@ -712,7 +739,9 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     geo.x_bytes = xb;
     geo.g_bytes = gb;
     geo.stage_bytes = (uint32_t)sb;
-    geo.tx_bytes = (uint32_t)((size_t)a.n * C * (8 + sizeof(GT)));
+    geo.m_off = xb;
+    geo.g_off = HAS_M ? 2 * xb : xb;
+    geo.tx_bytes = (uint32_t)((size_t)a.n * C * ((HAS_M ? 8 : 4) + sizeof(GT)));
     geo.tables_in_smem = tables_in_smem;
     geo.num_tiles = (a.d + C - 1) / C;
     size_t smem = fixed + (size_t)stages * sb;
@@ -819,7 +848,7 @@ int launch_rule(const dlm_step_args& a, cudaStream_t stream) {
         dlm_step_args b = a;
         b.d = a.d - d4;
         b.x = a.x + d4;
-        b.m = a.m + d4;
+        b.m = a.m ? a.m + d4 : nullptr;
         b.g = (const unsigned char*)a.g + d4 * sizeof(GT);
         rc = launch_tile<RULE, GT, 1>(b, stream);
     }
@@ -830,6 +859,12 @@ int launch_rule(const dlm_step_args& a, cudaStream_t stream) {
 
 int dlm_launch_step(int rule, const dlm_step_args& a, void* stream) {
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (rule == DLM_RULE_DSGD_ATC)
+        return a.g_dtype == DLM_G_BF16 ? launch_rule<DLM_RULE_DSGD_ATC, __nv_bfloat16>(a, s)
+                                       : launch_rule<DLM_RULE_DSGD_ATC, float>(a, s);
+    if (rule == DLM_RULE_DSGD_AWC)
+        return a.g_dtype == DLM_G_BF16 ? launch_rule<DLM_RULE_DSGD_AWC, __nv_bfloat16>(a, s)
+                                       : launch_rule<DLM_RULE_DSGD_AWC, float>(a, s);
     if (rule == DLM_RULE_DECENTLAM)
         return a.g_dtype == DLM_G_BF16 ? launch_rule<DLM_RULE_DECENTLAM, __nv_bfloat16>(a, s)
                                        : launch_rule<DLM_RULE_DECENTLAM, float>(a, s);

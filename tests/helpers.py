@@ -51,6 +51,8 @@ def to64(t):
 
 
 def oracle_rule(rule, W, x, m, g, beta, gamma, threads=THREADS):
+    if rule in ("dsgd_atc", "dsgd_awc"):
+        return oracle.dsgd_step(W, x, g, gamma, 0 if rule == "dsgd_atc" else 1, threads), m
     if rule == "decentlam":
         return oracle.decentlam_step(W, x, m, g, beta, gamma, threads)
     if rule == "dmsgd":
@@ -60,7 +62,9 @@ def oracle_rule(rule, W, x, m, g, beta, gamma, threads=THREADS):
 
 def lib_rule(rule, topo, k, x, m, g, beta, gamma):
     from paper_2104_11981_b200 import binding as B
-    if rule == "decentlam":
+    if rule in ("dsgd_atc", "dsgd_awc"):
+        B.dsgd_step(topo, k, x, g, gamma, B.DSGD_ATC if rule == "dsgd_atc" else B.DSGD_AWC)
+    elif rule == "decentlam":
         B.decentlam_step(topo, k, x, m, g, beta, gamma)
     elif rule == "dmsgd":
         B.dmsgd_step(topo, k, x, m, g, beta, gamma)

@@ -188,6 +188,13 @@ def test_step_argument_validation_on_host():
         assert step(fn, gamma=-0.1) == -5
         assert step(fn, beta=1.0) == -5 and step(fn, beta=-0.1) == -5 and step(fn, beta=float("nan")) == -5
         assert step(fn, gd=2) == -6
+    def dsgd(topo=t.handle, k=0, n=4, d=64, ld=64, x=X, g=G, gd=0, ldg=64, gamma=0.1, variant=0):
+        return lib.dsgd_step(topo, k, n, d, ld, vp(x), vp(g), gd, ldg, gamma, variant, None)
+
+    assert dsgd(topo=None) == -1 and dsgd(x=0) == -1 and dsgd(g=0) == -1
+    assert dsgd(n=0) == -2 and dsgd(ld=3) == -2 and dsgd(n=5) == -2 and dsgd(k=-2) == -2
+    assert dsgd(x=X + 1) == -3 and dsgd(g=X + 32) == -4 and dsgd(gamma=0.0) == -5
+    assert dsgd(gd=3) == -6 and dsgd(variant=2) == -6
     p = lambda **kw: lib.pmsgd_step(kw.get("n", 4), kw.get("d", 64), kw.get("ld", 64), vp(kw.get("x", X)),
                                     vp(kw.get("m", M)), vp(kw.get("g", G)), kw.get("gd", 0), kw.get("ldg", 64),
                                     kw.get("beta", 0.9), kw.get("gamma", 0.1), None)

@@ -354,3 +354,44 @@ def test_planted_mistakes_are_caught():
     assert not np.allclose(good[0], oracle.decentlam_step(W.T.copy(), x, m, g, 0.9, 0.1)[0])
     assert not np.allclose(good[0], oracle.decentlam_step(np.eye(8), x, m, g, 0.9, 0.1)[0])
     assert not np.allclose(good[0], oracle.decentlam_step(W, x, m, -g, 0.9, 0.1)[0])
+
+
+# --------------------------------------------------------------------------- DSGD without momentum
+@pytest.mark.parametrize("gname", list(_graphs()))
+def test_dsgd_variants_against_numpy(gname):
+    """Sec. 3 (adapt-then-combine): x' = W(x - gamma g); Remark in Sec. 5 (adapt-with-combine):
+    x' = W x - gamma g, both with numpy matmul on the exactly row-stochastic W."""
+    W = _graphs()[gname]; n = W.shape[0]
+    off = W.copy(); np.fill_diagonal(off, 0.0)
+    Wx = off + np.diag(1.0 - off.sum(1))
+    x, g = _rand(n, 6, 111), _rand(n, 6, 112)
+    np.testing.assert_allclose(oracle.dsgd_step(W, x, g, 0.1, 0), Wx @ (x - 0.1 * g), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(oracle.dsgd_step(W, x, g, 0.1, 1), Wx @ x - 0.1 * g, rtol=0, atol=1e-14)
+
+
+def test_dsgd_complete_graph_is_parallel_sgd():
+    """Sec. 3: fully connected with w_ij = 1/n, DSGD is parallel SGD: every row becomes xbar - gamma gbar."""
+    n, d = 4, 5
+    W = oracle.topology_dense(oracle.COMPLETE, n)
+    x, g = _rand(n, d, 121), _rand(n, d, 122)
+    out = oracle.dsgd_step(W, x, g, 0.25, 0)
+    np.testing.assert_allclose(out, np.tile(x.mean(0) - 0.25 * g.mean(0), (n, 1)), rtol=0, atol=1e-14)
+
+
+def test_dsgd_fixed_points_on_quadratics():
+    """On f_i(x) = ||x - c_i||^2 / 2 (grad = x - c): the ATC limit solves (I-W)X = -gamma W (X - C)
+    (the DecentLaM fixed point of App. C), the AWC limit solves (I-W)X = -gamma (X - C)."""
+    n, d, gamma = 8, 3, 0.2
+    W = oracle.topology_dense(oracle.RING, n)
+    off = W.copy(); np.fill_diagonal(off, 0.0)
+    Wx = off + np.diag(1.0 - off.sum(1)); L = np.eye(n) - Wx
+    C = _rand(n, d, 131)
+    for variant, M in ((0, Wx), (1, np.eye(n))):
+        x = np.zeros((n, d))
+        for _ in range(3000):
+            x = oracle.dsgd_step(W, x, x - C, gamma, variant)
+        want = np.linalg.solve(L + gamma * M, gamma * M @ C)
+        np.testing.assert_allclose(x, want, rtol=0, atol=1e-10)
+    # ATC equals DmSGD and DecentLaM at beta = 0 in x
+    x, g = _rand(n, d, 132), _rand(n, d, 133)
+    np.testing.assert_allclose(oracle.dsgd_step(W, x, g, gamma, 0), oracle.dmsgd_step(W, x, 0 * x, g, 0.0, gamma)[0], atol=0)
