@@ -266,6 +266,7 @@ DLM_API int dlm_kernel_error(int* flag);
  *           only; one staged value per neighbour)
  *   knob 8  lsq_grad: row chunks per node (at most 64)
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
+ *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
  * the default for DecentLaM on rows of 12 or more entries) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.

@@ -10,6 +10,8 @@
 
 #include "dlm_internal.h"
 
+int g_pmsgd_tune_cap = 0;  // blocks per SM of the grid, 0 = one block per 256 column groups
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -127,7 +129,7 @@ int launch(int n, int64_t d, int64_t ld, float* x, float* m, const GT* g, int64_
         return DLM_ERR_CUDA;
     long long groups = d / VEC;
     long long blocks = (groups + kThreads - 1) / kThreads;
-    long long cap = (long long)sms * 32;
+    long long cap = g_pmsgd_tune_cap > 0 ? (long long)sms * g_pmsgd_tune_cap : 0x7fffffffLL;
     if (blocks > cap) blocks = cap;
     pmsgd_kernel<GT, VEC><<<(unsigned)blocks, kThreads, 0, s>>>(n, d, ld, x, m, g, ldg, beta, gamma);
     dlm_count_launch(1);
