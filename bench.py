@@ -51,10 +51,10 @@ def parse_args():
 # SHA-256 matches, otherwise "traffic" is null.
 NCU_CAPTURE = {
     "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
-    "sha256": "f28533ba5eb2cf9b88f328d927d52440c287b2d5dfe5bb8c9568e3864ef0b0cc",
+    "sha256": "343a884036cde811ab4650f9d5b9fb2e33430e2f933022d7ecdddc9013700929",
     "workload": "cfg2",
-    "dram_read_bytes_per_np": 402.70e6 / (16 * 2097152),
-    "dram_write_bytes_per_np": 216.02e6 / (16 * 2097152),
+    "dram_read_bytes_per_np": 402.72e6 / (16 * 2097152),
+    "dram_write_bytes_per_np": 215.54e6 / (16 * 2097152),
 }
 
 
@@ -137,11 +137,14 @@ def dist_setup(n_gpus):
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world > 1:
+        import torch
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        import torch
-        backend = "nccl" if torch.cuda.is_available() else "gloo"
-        dist.init_process_group(backend=backend)
+        if torch.cuda.is_available():
+            torch.cuda.set_device(local)     # before the process group, so NCCL binds to this rank's GPU
+            dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend="gloo")
         return rank, world, local, dist
     return rank, world, local, None
 

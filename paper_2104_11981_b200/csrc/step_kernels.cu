@@ -270,9 +270,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 // CTA-wide bounded wait with a uniform result.  Only the first warp polls; the others sleep in the CTA
-// barrier instead of spending issue slots (ncu counted about 45 % of the pipeline kernel's warp
-// instructions in polling loops before).  After the barrier every other thread observes the completed
-// phase itself with a try_wait that returns at once, which makes the copies' writes visible to it.
+// barrier instead of spinning (6 % fewer warp instructions on the 16-node workload, same run time).
+// After the barrier every other thread observes the completed phase itself with a try_wait that
+// returns at once, which makes the copies' writes visible to it.
 __device__ __forceinline__ bool cta_wait(uint32_t bar, uint32_t parity) {
     bool ok = true;
     if (threadIdx.x < 32) ok = mbar_wait(bar, parity);
