@@ -130,7 +130,8 @@ DLM_API int topology_destroy(dlm_topology* topo);
 
 /* ------------------------------------------------------------------------------------
  * Update rules.  Common arguments:
- *   topo      : weights; slot k mod period is used.
+ *   topo      : weights; slot k mod period is used.  Its tables live on the GPU that was current when it
+ *               was built; calling with another GPU current fails with DLM_ERR_CUDA.
  *   k         : iteration counter (>= 0), only selects the slot.
  *   n, d      : nodes (must equal the topology's n) and coordinates per node.
  *   x, m      : device fp32 [n, d], row stride ld elements (ld >= d); updated IN PLACE.

@@ -59,6 +59,8 @@ int topo_step(int rule, const dlm_topology* topo, int64_t k, int n, int64_t d, i
     if (n != topo->n || k < 0) return DLM_ERR_SHAPE;
     const dlm_slot& s = topo->slots[(size_t)(k % (int64_t)topo->slots.size())];
     if (!s.d_rowptr) return DLM_ERR_CUDA;  // host-only handle
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != topo->device) return DLM_ERR_CUDA;  // tables live on another GPU
     dlm_step_args a;
     a.n = n;
     a.d = d;

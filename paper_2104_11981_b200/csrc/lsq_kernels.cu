@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
                                                                      const float* __restrict__ x,
                                                                      float* __restrict__ partial) {
     extern __shared__ __align__(16) unsigned char lsq_smem[];
+    // launched with programmatic stream serialization: x comes from the kernel before this one
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     unsigned char* base = lsq_smem + ((128u - (lsq_smem_u32(lsq_smem) & 127u)) & 127u);
     const uint32_t chunk_bytes = (uint32_t)kWarps * q * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)kStages * chunk_bytes);
@@ -196,6 +198,7 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
             if (threadIdx.x == 0) issue(st, c + kStages);
         }
     }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the reduction kernel may start launching
     __syncthreads();  // all stages consumed: reuse the first one for the cross-warp sum
     float* red = reinterpret_cast<float*>(base);
 #pragma unroll
@@ -254,8 +257,11 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_generic_kernel(int p, in
 }
 
 __global__ void __launch_bounds__(kThreads) lsq_reduce_kernel(int n, int q, int splits, float scale,
-                                                               const float* __restrict__ partial,
-                                                               float* __restrict__ g) {
+                                                               const float* partial, float* __restrict__ g) {
+    // Launched with programmatic stream serialization: its blocks may be scheduled while the
+    // partial-sum kernel drains; this wait returns once that whole grid has completed and its
+    // writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long e = (long long)blockIdx.x * kThreads + threadIdx.x;
     if (e >= (long long)n * q) return;
     const int i = (int)(e / q), c = (int)(e % q);
@@ -317,7 +323,17 @@ int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, con
         auto kern = lsq_partial_bulk_kernel<Q4>;                                                              \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
             return DLM_ERR_CUDA;                                                                              \
-        kern<<<grid, kThreads, smem, st>>>(p, q, rows, S, A, b, x, partial);                                  \
+        cudaLaunchConfig_t cfg = {};                                                                          \
+        cfg.gridDim = grid;                                                                                   \
+        cfg.blockDim = dim3(kThreads);                                                                        \
+        cfg.dynamicSmemBytes = smem;                                                                          \
+        cfg.stream = st;                                                                                      \
+        cudaLaunchAttribute attr[1];                                                                          \
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                      \
+        attr[0].val.programmaticStreamSerializationAllowed = 1;                                               \
+        cfg.attrs = attr;                                                                                     \
+        cfg.numAttrs = 1;                                                                                     \
+        if (cudaLaunchKernelEx(&cfg, kern, p, q, rows, S, A, b, x, partial) != cudaSuccess) return DLM_ERR_CUDA; \
     } break;
         switch (q / 128) {
             DLM_LSQ_BULK(1) DLM_LSQ_BULK(2) DLM_LSQ_BULK(3) DLM_LSQ_BULK(4)
@@ -341,9 +357,20 @@ int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, con
     }
     if (cudaGetLastError() != cudaSuccess) return DLM_ERR_CUDA;
     long long total = (long long)n * q;
-    lsq_reduce_kernel<<<(unsigned)((total + kThreads - 1) / kThreads), kThreads, 0, st>>>(n, q, S, scale, partial, g);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((total + kThreads - 1) / kThreads));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* partial_c = partial;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, lsq_reduce_kernel, n, q, S, scale, partial_c, g);
     dlm_count_launch(2);
-    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------

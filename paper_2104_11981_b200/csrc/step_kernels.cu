@@ -178,6 +178,11 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* gs = xs + (size_t)a.n * C;
     void* tab = (RULE == DLM_RULE_DECENTLAM) ? (void*)(gs + (size_t)a.n * C) : (void*)gs;
+    // This kernel serves the small, latency-bound problems and is launched with programmatic
+    // stream serialization: it may be scheduled while its predecessor drains and waits here until
+    // that grid has completed and its writes are visible (the tables never change, so staging
+    // them would be safe earlier, but they are tiny).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const Tables t = stage_tables(a, tab, tables_in_smem != 0);
     const GT* g = reinterpret_cast<const GT*>(a.g);
     const int items = a.n << cv_shift;
@@ -674,7 +679,7 @@ int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
     if (g_tune_cols >= VEC && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
     while ((long long)C / 2 >= a.d && C / 2 >= VEC) C /= 2;
     // small problems: prefer enough tiles to occupy every SM over wide tiles
-    while (C / 2 >= 32 * VEC && (a.d + C - 1) / C < dev.sms) C /= 2;
+    while (C / 2 >= 8 * VEC && (a.d + C - 1) / C < dev.sms) C /= 2;
     size_t tile_bytes = (size_t)a.n * C * 4 * arrays;
     if (tile_bytes + 16 > (size_t)dev.smem_optin) return DLM_ERR_UNSUPPORTED;
     int tables_in_smem = tile_bytes + table_bytes(a) + 16 <= (size_t)std::min(dev.smem_optin, 112 * 1024);
@@ -685,9 +690,19 @@ int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
         return DLM_ERR_CUDA;
     int per_sm = std::max(1, std::min(8, (int)((size_t)dev.smem_optin / (smem + 1024))));
     long long grid = std::min<long long>(num_tiles, (long long)dev.sms * per_sm);
-    kern<<<(unsigned)grid, kThreads, smem, stream>>>(a, C, ilog2(C / VEC), tables_in_smem, num_tiles);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kern, a, C, ilog2(C / VEC), tables_in_smem, (long long)num_tiles);
     dlm_count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
 // Returns DLM_OK if launched, DLM_ERR_UNSUPPORTED if this shape cannot use the pipeline kernel.
