@@ -161,6 +161,26 @@ DLM_API int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d
                    float beta, float gamma, void* cuda_stream);
 
 /*
+ * decentlam_step for gradients that still sit in HOST memory (this step's stochastic gradients as
+ * the data-parallel workers produced them): the same update, with the host-to-device transfer
+ * pipelined against the computation.  The columns are cut into chunks of chunk_cols; chunk j+1 is
+ * copied (on a library-owned copy stream) while chunk j is updated (on cuda_stream).  Every rule is
+ * coordinate-wise, so the result is bitwise that of decentlam_step on the whole array.
+ *   g_host     : host [n, d], row stride ldg elements; page-locked memory is needed for the copy to
+ *                overlap (pageable memory works but serialises); must stay valid until cuda_stream
+ *                has passed this call.
+ *   staging    : device scratch of 2 * n * chunk_cols * sizeof(element) bytes, 256-byte aligned, owned by
+ *                the caller; two calls sharing it must be ordered on the same stream.
+ *   chunk_cols : multiple of 8, at least 8 (a few million columns amortise the per-chunk launches).
+ * The first call on a device creates the copy stream and five events (kept until the process
+ * ends); make it outside any stream capture.  Other arguments and errors as for decentlam_step.
+ */
+DLM_API int decentlam_step_host_gradients(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
+                                          float* x, float* m, const void* g_host, int g_dtype, int64_t ldg,
+                                          void* staging, int64_t chunk_cols, float beta, float gamma,
+                                          void* cuda_stream);
+
+/*
  * DmSGD (Algorithm 1; App. A matrix form):
  *   m_i <- beta m_i + g_i ;  y_i = x_i - gamma m_i(new) ;
  *   x_i <- y_i + sum_{j in N_i, j != i} w_ij (y_j - y_i)      (= sum_j w_ij y_j for unit row sums)

@@ -52,6 +52,8 @@ for _name in ("topology_tables_host", "topology_tables_device"):
 _lib.topology_destroy.argtypes = [_vp]
 for _name in ("decentlam_step", "dmsgd_step"):
     getattr(_lib, _name).argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
+_lib.decentlam_step_host_gradients.argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _vp, _i64, _flt,
+                                               _flt, _vp]
 _lib.dsgd_step.argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _int, _i64, _flt, _int, _vp]
 _lib.pmsgd_step.argtypes = [_int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
 _lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
@@ -64,7 +66,7 @@ _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
 _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
-           "topology_tables_device", "topology_destroy", "decentlam_step", "dmsgd_step", "dsgd_step", "pmsgd_step",
+           "topology_tables_device", "topology_destroy", "decentlam_step", "decentlam_step_host_gradients", "dmsgd_step", "dsgd_step", "pmsgd_step",
            "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
@@ -185,6 +187,21 @@ def decentlam_step(topo, k, x, m, g, beta, gamma, stream=None):
     n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
     _check(_lib.decentlam_step(topo.handle, k, n, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)),
            "decentlam_step")
+
+
+def decentlam_step_host_gradients(topo, k, x, m, g_host, staging, chunk_cols, beta, gamma, stream=None):
+    """decentlam_step with g in (pinned) host memory: chunked copy overlapped with the update.
+    staging: device tensor of g's dtype with at least 2 * n * chunk_cols elements."""
+    import torch
+    assert not g_host.is_cuda and g_host.dim() == 2 and g_host.stride(1) == 1 and g_host.shape == x.shape
+    assert x.is_cuda and m.is_cuda and staging.is_cuda and staging.dtype == g_host.dtype
+    n, d = x.shape
+    assert staging.numel() >= 2 * n * chunk_cols and m.stride(0) == x.stride(0)
+    gd = G_F32 if g_host.dtype == torch.float32 else G_BF16
+    _check(_lib.decentlam_step_host_gradients(topo.handle, k, n, d, x.stride(0), _vp(x.data_ptr()), _vp(m.data_ptr()),
+                                              _vp(g_host.data_ptr()), gd, g_host.stride(0), _vp(staging.data_ptr()),
+                                              chunk_cols, beta, gamma, _stream_ptr(stream)),
+           "decentlam_step_host_gradients")
 
 
 def dmsgd_step(topo, k, x, m, g, beta, gamma, stream=None):

@@ -1,7 +1,9 @@
 // C ABI entry points: argument validation, slot selection, dispatch to the launchers.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
+#include <mutex>
 #include <cmath>
 #include <cstdint>
 
@@ -110,6 +112,84 @@ const char* dlm_status_string(int status) {
 int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, float* m,
                    const void* g, int g_dtype, int64_t ldg, float beta, float gamma, void* cuda_stream) {
     return topo_step(DLM_RULE_DECENTLAM, topo, k, n, d, ld, x, m, g, g_dtype, ldg, beta, gamma, cuda_stream);
+}
+
+namespace {
+
+// Copy stream and events of decentlam_step_host_gradients, one set per device, created on first use
+// and kept for the life of the process.
+struct HostFeed {
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copied[2] = {nullptr, nullptr};  // slot filled
+    cudaEvent_t freed[2] = {nullptr, nullptr};   // slot consumed by its kernel
+    cudaEvent_t ready = nullptr;                 // caller's stream reached the call
+    bool ok = false;
+};
+
+HostFeed* host_feed_for_current_device() {
+    static HostFeed feeds[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    HostFeed& f = feeds[dev];
+    if (!f.ok) {
+        if (cudaStreamCreateWithFlags(&f.copy_stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventCreateWithFlags(&f.copied[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&f.freed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+        if (cudaEventCreateWithFlags(&f.ready, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        f.ok = true;
+    }
+    return &f;
+}
+
+}  // namespace
+
+int decentlam_step_host_gradients(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x,
+                                  float* m, const void* g_host, int g_dtype, int64_t ldg, void* staging,
+                                  int64_t chunk_cols, float beta, float gamma, void* cuda_stream) {
+    if (!g_host || !staging) return DLM_ERR_NULL;
+    if (g_dtype != DLM_G_F32 && g_dtype != DLM_G_BF16) return DLM_ERR_KIND;
+    if (chunk_cols < 8 || chunk_cols % 8 != 0 || ldg < d) return DLM_ERR_SHAPE;
+    if ((uintptr_t)staging % 256) return DLM_ERR_ALIGN;
+    const size_t esz = g_dtype == DLM_G_BF16 ? 2 : 4;
+    const size_t slot_bytes = (size_t)n * chunk_cols * esz;
+    // validate everything else once, against the first staging slot standing in for g
+    {
+        int rc = check_state(n, std::min<int64_t>(d, chunk_cols), ld, x, m, staging, g_dtype, chunk_cols, beta, gamma);
+        if (rc != DLM_OK) return rc;
+        if (n < 1 || d < 1 || ld < d) return DLM_ERR_SHAPE;
+        Range rs = {(uintptr_t)staging, (uintptr_t)staging + 2 * slot_bytes};
+        if (overlap(rs, span(x, n, d, ld, 4)) || overlap(rs, span(m, n, d, ld, 4))) return DLM_ERR_ALIAS;
+    }
+    if (!topo) return DLM_ERR_NULL;
+    HostFeed* f = host_feed_for_current_device();
+    if (!f) return DLM_ERR_CUDA;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // the first copies may overwrite slots only after earlier work of the caller's stream (a previous
+    // call's kernels) has been ordered before them
+    if (cudaEventRecord(f->ready, stream) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaStreamWaitEvent(f->copy_stream, f->ready, 0) != cudaSuccess) return DLM_ERR_CUDA;
+    int64_t chunk = 0;
+    for (int64_t c0 = 0; c0 < d; c0 += chunk_cols, ++chunk) {
+        const int slot = (int)(chunk & 1);
+        const int64_t cols = std::min<int64_t>(chunk_cols, d - c0);
+        unsigned char* dst = static_cast<unsigned char*>(staging) + (size_t)slot * slot_bytes;
+        if (chunk >= 2 && cudaStreamWaitEvent(f->copy_stream, f->freed[slot], 0) != cudaSuccess) return DLM_ERR_CUDA;
+        if (cudaMemcpy2DAsync(dst, (size_t)chunk_cols * esz, static_cast<const unsigned char*>(g_host) + (size_t)c0 * esz,
+                              (size_t)ldg * esz, (size_t)cols * esz, (size_t)n, cudaMemcpyHostToDevice,
+                              f->copy_stream) != cudaSuccess)
+            return DLM_ERR_CUDA;
+        if (cudaEventRecord(f->copied[slot], f->copy_stream) != cudaSuccess) return DLM_ERR_CUDA;
+        if (cudaStreamWaitEvent(stream, f->copied[slot], 0) != cudaSuccess) return DLM_ERR_CUDA;
+        int rc = topo_step(DLM_RULE_DECENTLAM, topo, k, n, cols, ld, x + c0, m + c0, dst, g_dtype, chunk_cols, beta, gamma,
+                           cuda_stream);
+        if (rc != DLM_OK) return rc;
+        if (cudaEventRecord(f->freed[slot], stream) != cudaSuccess) return DLM_ERR_CUDA;
+    }
+    return DLM_OK;
 }
 
 int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld, float* x, float* m,
