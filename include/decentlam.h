@@ -247,8 +247,8 @@ DLM_API int lsq_grad(int n, int p, int q, const float* A, const float* b, const 
  * same g), minus the workspace.  Neither this call nor anything below it calls cudaMalloc,
  * cudaFree or an allocating library routine.
  *   - Size limit: n * S * q * 4 bytes must fit the array, S <= 64 being the number of row chunks
- *     per node the library picks for (n, p) on the current GPU (about 2 * SM count / n).  The cfg4
- *     problem (n = 32, q = 1024) needs 1.2 MiB.  Larger problems return DLM_ERR_WORKSPACE and
+ *     per node the library picks for (n, p) on the current GPU (about 2 * SM count / n).  A problem
+ *     with n = 32 nodes, p = 4096 and q = 1024 needs 1.2 MiB.  Larger problems return DLM_ERR_WORKSPACE and
  *     launch nothing; use lsq_grad with your own workspace instead.
  *   - First call on a device: looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current) and caches it; make this first call outside any stream capture.
