@@ -133,3 +133,28 @@ def test_cfg5_general_csr_sampled(rule):
 
 def test_cfg5_consensus_start():
     _sampled_run("cfg5", "decentlam", True, n_random=1024, steps=10)
+
+
+@pytest.mark.parametrize("cfg", ["cfg2", "cfg3", "cfg5"])
+def test_node_average_invariant_on_full_tensors(cfg):
+    """App. D: because the columns of W sum to one, the node average obeys
+    mbar' = beta mbar + gbar, xbar' = xbar - gamma mbar' for DecentLaM and DmSGD.  Checked on the
+    whole [n, d] state at the workload's full size (a property that needs no oracle run); the
+    averages are formed in fp64 with torch reductions, which are not part of the product."""
+    w = WORKLOADS[cfg]; dev = torch.device("cuda:0")
+    topo, _ = build_both(w.topology, w.n, graph_seed=seed_for(cfg, inputs.P_GRAPH), er_p=w.er_p or 0.05)
+    gt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    for rule in ("decentlam", "dmsgd"):
+        x = inputs.normal_torch((w.n, w.d), w.x0_std, seed_for(cfg, inputs.P_X0), dev)
+        m = inputs.normal_torch((w.n, w.d), 1e-3, seed_for(cfg, 9), dev)
+        for k in range(3):
+            g = inputs.normal_torch((w.n, w.d), w.g_std, seed_for(cfg, inputs.P_G0 + k), dev, dtype=gt)
+            xbar, mbar, gbar = (t.double().mean(0) for t in (x, m, g.float()))
+            lib_rule(rule, topo, k, x, m, g, w.beta, w.gamma)
+            mbar_want = float(np.float32(w.beta)) * mbar + gbar
+            xbar_want = xbar - float(np.float32(w.gamma)) * mbar_want
+            # fp32 rounding of n values per column, averaged: a few 1e-8 relative to the largest entries
+            em = (m.double().mean(0) - mbar_want).abs().max().item() / m.abs().max().item()
+            ex = (x.double().mean(0) - xbar_want).abs().max().item() / x.abs().max().item()
+            assert em <= 2e-7 and ex <= 2e-7, (cfg, rule, k, em, ex)
+            del g
