@@ -283,13 +283,13 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 4  tiles per CTA: t > 0 launches ceil(tiles / t) CTAs; t < 0 a persistent grid
  *   knob 5  neighbour tables: 1 = staged in shared memory, 2 = read from global memory
  *   knob 6  threads per CTA of the pipeline kernels (128, 256 or 512)
- *   knob 7  1 = pipeline kernel with the plain mixing loop, 2 = merged-staging kernel (DecentLaM
- *           only; one staged value per neighbour)
+ *   knob 7  1 = pipeline kernel with the plain mixing loop, 2 = merged-staging kernel (one staged
+ *           value per neighbour)
  *   knob 8  lsq_grad: row chunks per node (at most 64)
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
  *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
- * the default for DecentLaM on rows of 12 or more entries) arranges the same sum differently and
+ * the default on rows of 12 or more entries) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);

@@ -78,6 +78,7 @@ int topo_step(int rule, const dlm_topology* topo, int64_t k, int n, int64_t d, i
     a.order = s.d_order;
     a.rows = s.d_rows;
     a.ent = s.d_ent;
+    a.selfw = s.d_selfw;
     a.nnz = (int)s.col.size();
     a.max_degree = s.max_degree;
     a.beta = beta;

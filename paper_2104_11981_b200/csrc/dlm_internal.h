@@ -14,8 +14,10 @@ struct dlm_slot {
     // packed copies for the warp-cooperative kernels: rows[r] = {i, first entry, length, bits of S_i = sum_j w_ij} in
     // processing order; ent[p] = {col[p], bits of val[p]}
     std::vector<int32_t> rows, ent;
+    std::vector<int32_t> selfw;  // per row in processing order: bits of (float)(1 - sum_{j != i} w_ij)
     int32_t* d_rows = nullptr;
     int32_t* d_ent = nullptr;
+    int32_t* d_selfw = nullptr;
     int32_t* d_rowptr = nullptr;
     int32_t* d_col = nullptr;
     float* d_val = nullptr;
@@ -45,6 +47,7 @@ struct dlm_step_args {
     const int32_t* order;   // device, row processing order (a permutation of 0..n-1)
     const int32_t* rows;    // device, int4 per row in processing order {i, first entry, length, bits of S_i}
     const int32_t* ent;     // device, int2 per entry {col, bits of val}
+    const int32_t* selfw;   // device, per row in processing order: bits of the exact self weight 1 - sum_{j != i} w_ij
     int nnz;
     int max_degree;
     float beta, gamma, inv_gamma;

@@ -431,20 +431,24 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
 
 
 // ---------------------------------------------------------------------------------------------
-// Merged-staging DecentLaM kernel for long neighbour lists (many nodes, dense rows).
+// Merged-staging kernel for long neighbour lists (many nodes, dense rows): ONE staged value per
+// neighbour, a branch-free weighted sum over the row, two float4 column groups per thread.
 //
-// With z_j = x_j - r (r = row 0's value of the column: a common reference that keeps z small
-// whenever the replicas are close) and v_j = g_j - z_j / gamma, Eq. (decentLaM-x-1) reads
+// DecentLaM.  With z_j = x_j - r (r = row 0's value of the column: a common reference that keeps z
+// small whenever the replicas are close) and v_j = g_j - z_j / gamma, Eq. (decentLaM-x-1) reads
 //     g~_i = sum_{j in N_i} w_ij v_j + z_i S_i / gamma,      S_i = sum_{j != i} w_ij + w_ii (stored),
 // (expand: sum_j w_ij g_j + (1/gamma) sum_{j != i} w_ij (z_i - z_j); the self term of the v-sum
-// cancels against w_ii z_i / gamma).  So ONE staged value per neighbour, no subtraction and no
-// self special case in the loop.  Pass 1 turns the staged (x, g) into v: in place of g for fp32
-// gradients, in a tile of its own for bf16.  Pass 2: a thread owns two float4 column groups of a
-// row, the L = C/8 lanes that share the row fetch its table entries together and hand them round
-// with shuffles; slots past the end of a row carry weight 0 and point at row i itself, so the
-// loop is branch-free.  m is not staged: each thread reads its own m from global memory while
-// the loop runs.  Tables live in shared memory when they fit (the large shared-memory carve-out
-// leaves too little L1 to keep them cached otherwise).
+// cancels against w_ii z_i / gamma).  Pass 1 turns the staged (x, g) into v: in place of g for fp32
+// gradients, in a tile of its own for bf16; m is not staged, each thread reads its own m from
+// global memory while the loop runs.
+// DmSGD / DSGD.  The partial average sum_j w_ij y_j is taken as such, the self weight being the
+// exact remainder 1 - sum_{j != i} w_ij (rounded once to fp32).  Pass 1 forms y in place of x
+// (DmSGD: m' = beta m + g with m straight from global memory, y = x - gamma m'; adapt-then-combine:
+// y = x - gamma g; adapt-with-combine: y = x, no pass 1).
+// Pass 2: the L = C/8 lanes that share a row fetch its table entries together and hand them round
+// with shuffles; slots past the end of a row carry weight 0 and point at row i itself.  Tables live
+// in shared memory when they fit (the large shared-memory carve-out leaves too little L1 to keep
+// them cached otherwise).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ float4 lds128(uint32_t addr) {
     float4 v;
@@ -460,16 +464,17 @@ struct MergedGeom {
     int cv_shift;   // log2(C / 4)
     int tables_in_smem;
     uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
-    uint32_t v_off, g_off; // byte offsets of the v tile and of the g landing area inside the stage
+    uint32_t v_off, g_off; // byte offsets of the staged-value tile and of the g landing area inside the stage
     uint32_t stage_bytes;
     uint32_t tx_bytes;
     long long num_tiles;
 };
 
-template <typename GT>
+template <int RULE, typename GT>
 __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                            const __grid_constant__ CUtensorMap tm_g,
                                                            dlm_step_args a, MergedGeom geo) {
+    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char* st = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
     uint64_t* bar_ptr = reinterpret_cast<uint64_t*>(st + geo.stage_bytes);
@@ -501,8 +506,8 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
     }
     __syncthreads();
 
-    const float* xs = reinterpret_cast<const float*>(st);
-    float* vs = reinterpret_cast<float*>(st + geo.v_off);
+    float* xs = reinterpret_cast<float*>(st);
+    float* vs = reinterpret_cast<float*>(st + geo.v_off);  // staged values: v (DecentLaM) or y (the x tile itself)
     const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off);
     const int items = a.n << geo.cv_shift;
     const int cv_mask = (1 << geo.cv_shift) - 1;
@@ -518,38 +523,60 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
             return;                          // single stage: no other copy of this CTA is in flight
         }
         const long long tile_base = (first + it * gridDim.x) * C;
-        // pass 1: v = g - (x - r) / gamma
-        for (int e = threadIdx.x; e < items; e += blockDim.x) {
-            const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
-            const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
-            const Pack<4> gi = ld_g<4>(gs + i * C + off);
-            Pack<4> v;
+        if (RULE != DLM_RULE_DSGD_AWC) {  // pass 1 (the adapt-with-combine rule averages x as it is)
+            for (int e = threadIdx.x; e < items; e += blockDim.x) {
+                const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+                const Pack<4> xi = ld_f32<4>(xs + i * C + off);
+                const Pack<4> gi = ld_g<4>(gs + i * C + off);
+                Pack<4> v;
+                if (LAM) {  // v = g - (x - r) / gamma
+                    const Pack<4> ref = ld_f32<4>(xs + off);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
-            st_f32<4>(vs + i * C + off, v);
+                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
+                } else if (RULE == DLM_RULE_DMSGD) {  // m' = beta m + g ; y = x - gamma m'
+                    const long long c = tile_base + off;
+                    Pack<4> mi = {{0.f, 0.f, 0.f, 0.f}}, mn;
+                    if (c < a.d) mi = ld_f32<4>(a.m + (size_t)i * a.ld + c);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], v.v[u]);
+                    if (c < a.d) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                } else {  // adapt-then-combine: y = x - gamma g
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.gamma, gi.v[u], xi.v[u]);
+                }
+                st_f32<4>(vs + i * C + off, v);
+            }
+            __syncthreads();
         }
-        __syncthreads();
         // pass 2
         for (int e = threadIdx.x; e < witems_padded; e += blockDim.x) {
             const bool live = e < witems;
-            const int4 ri = rows[live ? (e >> lshift) : 0];
+            const int slot = live ? (e >> lshift) : 0;
+            const int4 ri = rows[slot];
             const int i = ri.x, len = ri.z;
             // column groups {q, q + L}; with four lanes per row, neighbouring rows take the two
             // halves in opposite order so that a quarter warp still covers all 32 banks
-            const int par = (L == 4) ? ((e >> lshift) & 1) : 0;
+            const int par = (L == 4) ? (slot & 1) : 0;
             const int off0 = (L == 4 ? glane + 4 * par : glane) * 4;
             const int off1 = (L == 4 ? glane + 4 * (1 - par) : glane + L) * 4;
             const long long c0 = tile_base + off0, c1 = tile_base + off1;
             const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;
             Pack<4> m0 = {{0.f, 0.f, 0.f, 0.f}}, m1 = {{0.f, 0.f, 0.f, 0.f}};
-            if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
-            if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            if (LAM) {
+                if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
+                if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            }
+            // the averaging rules replace the stored diagonal by the exact remainder 1 - sum_{j != i} w_ij
+            const int self_bits = LAM ? 0 : a.selfw[slot];
             float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t vb0 = smem_u32(vs) + off0 * 4, vb1 = smem_u32(vs) + off1 * 4;
             const int len_max = __reduce_max_sync(full, len);
             for (int base0 = 0; base0 < len_max; base0 += L) {
-                int2 en = make_int2(i, 0);  // filler: adds exactly 0 * v_i
-                if (base0 + glane < len) en = ent[ri.y + base0 + glane];
+                int2 en = make_int2(i, 0);  // filler: adds exactly 0 * (staged value of row i)
+                if (base0 + glane < len) {
+                    en = ent[ri.y + base0 + glane];
+                    if (!LAM && en.x == i) en.y = self_bits;
+                }
                 const int cnt = min(L, (len_max - base0 + 3) & ~3);
 #pragma unroll 4
                 for (int r = 0; r < cnt; ++r) {
@@ -567,18 +594,27 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int off = h ? off1 : off0;
-                const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
-                Pack<4> mn, xn;
+                Pack<4> xn;
+                if (LAM) {
+                    const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
+                    Pack<4> mn;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, h ? acc1[u] : acc0[u]);
-                    mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
-                    xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
+                    for (int u = 0; u < 4; ++u) {
+                        const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, h ? acc1[u] : acc0[u]);
+                        mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
+                        xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
+                    }
+                    if (h ? st1 : st0) st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) xn.v[u] = h ? acc1[u] : acc0[u];
+                    if (RULE == DLM_RULE_DSGD_AWC) {
+                        const Pack<4> gi = ld_g<4>(gs + i * C + off);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
+                    }
                 }
-                if (h ? st1 : st0) {
-                    st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
-                    st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
-                }
+                if (h ? st1 : st0) st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
             }
         }
         if (it + 1 < my_tiles) {
@@ -782,11 +818,12 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// DecentLaM with merged staging (long rows).  DLM_ERR_UNSUPPORTED if the shape does not fit.
-template <typename GT>
+// Merged staging (long rows).  DLM_ERR_UNSUPPORTED if the shape does not fit.
+template <int RULE, typename GT>
 int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     const DeviceInfo& dev = device_info();
     if (!dev.ok) return DLM_ERR_CUDA;
+    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
     const bool bf16 = sizeof(GT) == 2;
     if (a.n > 256 || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
     int C = 1 << ilog2(std::max(1, (int)(32768 / ((size_t)a.n * 4))));
@@ -800,10 +837,16 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
         const size_t xb = ((size_t)a.n * C * 4 + 127) & ~(size_t)127;
         const size_t gb = ((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127;
         geo.x_bytes = (uint32_t)xb;
-        geo.v_off = (uint32_t)xb;                       // fp32: v overwrites g in place
-        geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);     // bf16: g lands behind the v tile
-        geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
-        // tables in shared memory if two CTAs per SM still fit, or if one CTA fits and they are large
+        if (LAM) {  // [x | v | g]: for fp32 gradients v overwrites g in place
+            geo.v_off = (uint32_t)xb;
+            geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);
+            geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
+        } else {    // [x (becomes y) | g]
+            geo.v_off = 0;
+            geo.g_off = (uint32_t)xb;
+            geo.stage_bytes = (uint32_t)(xb + gb);
+        }
+        // tables in shared memory if two CTAs per SM still fit, or on request
         const size_t fixed = 128 + 16 + 16;
         const size_t with_tab = fixed + geo.stage_bytes + tab;
         geo.tables_in_smem = g_tune_tables == 2 ? 0 : (with_tab <= (size_t)dev.smem_optin / 2 - 1024 || g_tune_tables == 1);
@@ -817,7 +860,7 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     CUtensorMap tm_x, tm_g;
     if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, C) || !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, C))
         return DLM_ERR_UNSUPPORTED;
-    auto kern = step_merged_kernel<GT>;
+    auto kern = step_merged_kernel<RULE, GT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DLM_ERR_CUDA;
     const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : (geo.tables_in_smem ? 8 : 4);
@@ -828,14 +871,14 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// DecentLaM on rows of 12 or more entries takes the merged-staging kernel when the shape allows
-// it (measured on B200 at n = 256: 9-entry rows are faster with the plain loop, ~14-entry rows with
-// merged staging); everything else the pipeline kernel with the plain mixing loop.
+// Rows of 12 or more entries take the merged-staging kernel when the shape allows it (measured on
+// B200 at n = 256: 9-entry rows are faster with the plain loop, ~14-entry rows with merged staging);
+// everything else the pipeline kernel with the plain mixing loop.
 template <int RULE, typename GT>
 int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : a.max_degree >= 12;
-    if (merged && RULE == DLM_RULE_DECENTLAM) {
-        int rc = launch_merged<GT>(a, stream);
+    if (merged) {
+        int rc = launch_merged<RULE, GT>(a, stream);
         if (rc != DLM_ERR_UNSUPPORTED) return rc;
     }
     return launch_tma_plain<RULE, GT>(a, stream);

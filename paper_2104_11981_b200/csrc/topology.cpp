@@ -69,6 +69,7 @@ void make_order(dlm_slot& s) {
         return s.rowptr[a + 1] - s.rowptr[a] > s.rowptr[b + 1] - s.rowptr[b];
     });
     s.rows.resize((size_t)4 * n);
+    s.selfw.resize(n);
     for (int r = 0; r < n; ++r) {
         const int i = s.order[r];
         s.rows[4 * r + 0] = i;
@@ -78,6 +79,11 @@ void make_order(dlm_slot& s) {
         for (int32_t p = s.rowptr[i]; p < s.rowptr[i + 1]; ++p) row_sum += (double)s.val[p];
         const float S_i = (float)row_sum;
         std::memcpy(&s.rows[4 * r + 3], &S_i, sizeof(float));
+        double off_sum = 0.0;  // exact self weight of the averaging rules: 1 - sum_{j != i} w_ij, rounded once
+        for (int32_t p = s.rowptr[i]; p < s.rowptr[i + 1]; ++p)
+            if (s.col[p] != i) off_sum += (double)s.val[p];
+        const float self_w = (float)(1.0 - off_sum);
+        std::memcpy(&s.selfw[r], &self_w, sizeof(float));
     }
     s.ent.resize(2 * s.col.size());
     for (size_t p = 0; p < s.col.size(); ++p) {
@@ -94,6 +100,9 @@ int upload(dlm_slot& s) {
     if (cudaMemcpy(s.d_rows, s.rows.data(), s.rows.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return DLM_ERR_CUDA;
     if (cudaMemcpy(s.d_ent, s.ent.data(), s.ent.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return DLM_ERR_CUDA;
+    if (cudaMalloc((void**)&s.d_selfw, s.selfw.size() * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
+    if (cudaMemcpy(s.d_selfw, s.selfw.data(), s.selfw.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return DLM_ERR_CUDA;
     if (cudaMalloc((void**)&s.d_order, s.order.size() * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
     if (cudaMemcpy(s.d_order, s.order.data(), s.order.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
@@ -356,6 +365,7 @@ int topology_destroy(dlm_topology* topo) {
         if (s.d_order) cudaFree(s.d_order);
         if (s.d_rows) cudaFree(s.d_rows);
         if (s.d_ent) cudaFree(s.d_ent);
+        if (s.d_selfw) cudaFree(s.d_selfw);
         if (s.d_rowptr) cudaFree(s.d_rowptr);
         if (s.d_col) cudaFree(s.d_col);
         if (s.d_val) cudaFree(s.d_val);
