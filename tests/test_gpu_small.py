@@ -227,3 +227,13 @@ def test_topology_device_tables_exist():
     rowptr, col, val = topo.tables_host(0)
     rp, cp, vp, nnz = topo.tables_device(0)
     assert nnz == len(col) and rp and cp and vp
+
+
+@pytest.mark.parametrize("rule", ["decentlam", "dmsgd"])
+@pytest.mark.parametrize("n,topology,d", [(2048, "ring", 72), (512, "complete", 260), (256, "complete", 4100),
+                                           (1, "complete", 5000), (2, "static_exp", 100_003)])
+def test_extreme_node_counts(rule, n, topology, d):
+    """The largest supported n (tile kernel, tables in global memory), dense rows far beyond what
+    fits in shared memory (complete graphs: 256 or 512 entries per row), and the degenerate n = 1
+    (W = [1]: plain momentum SGD) and n = 2."""
+    _case(rule, topology, n, d, "f32", seed=n + d, steps=2)
