@@ -250,6 +250,13 @@ def time_steps(step_fn, reset_fn, steps, warmup, torch, stream, count_fn=lambda:
 def run_ours(args):
     import torch
 
+    from paper_2104_11981_b200 import build as lib_build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        lib_build.build()                            # no-op when libdecentlam.so is up to date; raises if nvcc fails
+    else:                                            # the other ranks of the node wait for rank 0's build
+        t_wait = time.time()
+        while lib_build._stale() and time.time() - t_wait < 300:
+            time.sleep(1.0)
     from paper_2104_11981_b200 import binding as B   # fails loudly if the CUDA library is missing
     from paper_2104_11981_b200 import inputs
     if not torch.cuda.is_available():

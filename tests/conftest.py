@@ -10,6 +10,12 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # The shared libraries are build outputs, not tracked files: (re)build them when missing or stale
+    # (nvcc cross-compiles without a GPU; a few seconds when nothing changed).
+    from paper_2104_11981_b200 import build as lib_build
+    lib_build.build()
+    from oracle import build as oracle_build
+    oracle_build.build()
 
 
 def pytest_collection_modifyitems(config, items):
