@@ -173,7 +173,8 @@ DLM_API int decentlam_step(const dlm_topology* topo, int64_t k, int n, int64_t d
  *                the caller; two calls sharing it must be ordered on the same stream.
  *   chunk_cols : multiple of 8, at least 8 (a few million columns amortise the per-chunk launches).
  * The first call on a device creates the copy stream and five events (kept until the process
- * ends); make it outside any stream capture.  Other arguments and errors as for decentlam_step.
+ * ends); make it outside any stream capture.  The stream and events are shared by all calls on that
+ * device: call it from one host thread at a time per device.  Other arguments and errors as for decentlam_step.
  */
 DLM_API int decentlam_step_host_gradients(const dlm_topology* topo, int64_t k, int n, int64_t d, int64_t ld,
                                           float* x, float* m, const void* g_host, int g_dtype, int64_t ldg,
