@@ -192,7 +192,13 @@ def oracle_sample(workload, budget_s=20.0):
         k += 1
     times.sort()
     med = times[len(times) // 2]
+    single = []
+    for k in range(2):                      # the same oracle on one thread, for the per-core figure
+        t0 = time.perf_counter()
+        oracle.decentlam_step(Ws[k % period], x, m, g, np.float32(w.beta), np.float32(w.gamma), 1)
+        single.append(time.perf_counter() - t0)
     return {"value": w.n * cols / med, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "single_thread_value": w.n * cols / min(single),
             "sample": f"{workload}: {len(times)} DecentLaM steps of the double-precision dense-W oracle on a "
                       f"[{w.n} x {cols}] column slab (median), {threads} threads"}, med, w.n * cols
 
@@ -307,6 +313,20 @@ def run_ours(args):
     value = job_units / job_secs
     peak, peak_kind = measured_peak()
     achieved = bytes_per_np * n * d * args.steps / secs / 1e9
+    # context only: a plain device copy timed in this very run (the roofline denominator stays the
+    # measured figure)
+    copy_gbs = None
+    if world == 1:
+        src = torch.empty(1 << 29, dtype=torch.float32, device=dev); dst = torch.empty_like(src)
+        for _ in range(2):
+            dst.copy_(src)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(stream)
+        for _ in range(5):
+            dst.copy_(src)
+        c1.record(stream); c1.synchronize()
+        copy_gbs = 2 * src.numel() * 4 * 5 / (c0.elapsed_time(c1) * 1e-3) / 1e9
+        del src, dst
 
     extra = {}
     if not args.no_extra and world == 1:
@@ -369,7 +389,8 @@ def run_ours(args):
                        "l2": f"working set {(8 + g.element_size()) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(args.workload, n * d), "peak_kind": f"of {peak_kind}",
-                         "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d},
+                         "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d,
+                         "copy_gbs_this_run": copy_gbs},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "cpu_baseline": cpu_baseline,
             "other_rules": extra,
         }
