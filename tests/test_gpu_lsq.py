@@ -161,3 +161,23 @@ def test_paper_linear_regression_setting():
     assert dm[2] > 2.0 * dsgd[2]                            # ... but DmSGD ends with the larger bias
     assert abs(lam[2] - dsgd[2]) <= 0.05 * dsgd[2]         # DecentLaM ends at DSGD's bias
     assert dm[2] / lam[2] <= 1.0 / (1.0 - beta) ** 2 * 1.01
+
+
+def test_lsq_kernel_variants_agree_bitwise():
+    """The bulk-copy pipeline kernel and the register-pipelined kernel sum in the same order; the
+    number of row chunks per node changes the order of the final sum only (rounding-level)."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    n, p, q = 6, 700, 512
+    A, b, _ = inputs.lsq_problem_torch(n, p, q, 31, dev)
+    x = inputs.normal_torch((n, q), 1.0, 32, dev)
+    try:
+        g_bulk = _lsq_gpu(A, b, x, 1.0 / p)
+        B.set_tuning(9, 2)
+        g_regs = _lsq_gpu(A, b, x, 1.0 / p)
+        assert torch.equal(g_bulk, g_regs)
+        B.set_tuning(9, 0); B.set_tuning(8, 3)
+        g_three = _lsq_gpu(A, b, x, 1.0 / p)
+        assert rel_l2(to64(g_three), to64(g_bulk)) <= 1e-6
+    finally:
+        B.set_tuning(8, 0); B.set_tuning(9, 0)
