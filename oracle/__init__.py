@@ -9,7 +9,9 @@ Pinned by tests/test_oracle_*.py (``-m "not gpu"``) against: the hand example fo
 Algorithms 1 and 2, weight-matrix invariants (Assumption A.3), the node-average recursion
 (App. D), the complete-graph and beta = 0 reductions (Sec. 3), the momentum-free
 reformulations (App. B), the s-domain recursion (Sec. 5), exact rational brute force, the
-fixed-point equations (App. C), finite differences and a library least-squares solve.
+fixed-point equations (App. C), finite differences and a library least-squares solve; the
+expanded (Gram) form of the least-squares gradient against the residual form, a hand example and
+pure-Python sums.
 """
 import ctypes
 import os
@@ -157,6 +159,33 @@ def lsq_grad(A, b, x, scale, threads=1):
     fp = ctypes.POINTER(ctypes.c_float)
     _L().orc_lsq_grad(n, p, q, A.ctypes.data_as(fp), b.ctypes.data_as(fp), _p(x), float(scale), _p(g), int(threads))
     return g
+
+
+def lsq_gram(A, b, scale):
+    """Expanded form of the same gradient (App. G objective): A^T(Ax - b) = (A^T A)x - A^T b.
+    Returns H [n,q,q] = scale * A_i^T A_i and c [n,q] = scale * A_i^T b_i in float64 (numpy matmul)."""
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    b = np.ascontiguousarray(b, dtype=np.float32)
+    n, p, q = A.shape
+    H = np.empty((n, q, q), dtype=np.float64)
+    c = np.empty((n, q), dtype=np.float64)
+    for i in range(n):
+        Ai = A[i].astype(np.float64)
+        H[i] = float(scale) * (Ai.T @ Ai)
+        c[i] = float(scale) * (Ai.T @ b[i].astype(np.float64))
+    return H, c
+
+
+def lsq_gram_entries(A, b, scale, node, rows, cols):
+    """Single entries H[node, rows[t], cols[t]] of lsq_gram, each as one float64 dot product of two
+    columns of A (for sampled checks at sizes where the whole of H is too slow on the CPU)."""
+    Ai = np.asarray(A[node], dtype=np.float64)
+    return np.array([float(scale) * float(Ai[:, r] @ Ai[:, c]) for r, c in zip(rows, cols)], dtype=np.float64)
+
+
+def lsq_grad_gram(H, c, x):
+    """g_i = H_i x_i - c_i in float64."""
+    return np.einsum("irc,ic->ir", _d(H), _d(x)) - _d(c)
 
 
 def lsq_optimum(A, b):

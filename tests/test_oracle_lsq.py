@@ -35,6 +35,39 @@ def test_lsq_grad_matches_numpy_and_threads():
     assert np.array_equal(g, oracle.lsq_grad(A, b, x, 1.0 / 50, threads=3))
 
 
+def test_lsq_gram_hand_example():
+    """A = [[1,2],[3,4]], b = (1,1), scale = 1/2: A^T A = [[10,14],[14,20]], A^T b = (4,6)."""
+    A = np.array([[[1, 2], [3, 4]]], dtype=np.float32)
+    b = np.array([[1, 1]], dtype=np.float32)
+    H, c = oracle.lsq_gram(A, b, 0.5)
+    assert np.array_equal(H[0], np.array([[5.0, 7.0], [7.0, 10.0]]))
+    assert np.array_equal(c[0], np.array([2.0, 3.0]))
+    # gradient at x = (1, -1): A x - b = (-2, -2); A^T r / 2 = (-4, -6)
+    assert np.array_equal(oracle.lsq_grad_gram(H, c, np.array([[1.0, -1.0]])), np.array([[-4.0, -6.0]]))
+
+
+def test_lsq_gram_agrees_with_residual_form_and_brute_force():
+    """H x - c equals the residual-form gradient (an independent loop nest in the C++ oracle); every
+    entry of H and c equals a pure-Python sum over rows; H is symmetric with trace scale*||A||_F^2."""
+    A, b, _ = _problem(3, 11, 6, seed=17)
+    scale = 1.0 / 11
+    H, c = oracle.lsq_gram(A, b, scale)
+    x = inputs.normal_np((3, 6), 1.0, 18).astype(np.float64)
+    g = oracle.lsq_grad(A, b, x, scale)
+    np.testing.assert_allclose(oracle.lsq_grad_gram(H, c, x), g, rtol=1e-12, atol=1e-13)
+    for i in range(3):
+        for r in range(6):
+            cr = sum(float(A[i, a, r]) * float(b[i, a]) for a in range(11)) * scale
+            assert abs(c[i, r] - cr) < 1e-14 * (1 + abs(cr))
+            for s in range(6):
+                hs = sum(float(A[i, a, r]) * float(A[i, a, s]) for a in range(11)) * scale
+                assert abs(H[i, r, s] - hs) < 1e-14 * (1 + abs(hs))
+        assert np.array_equal(H[i], H[i].T)
+        assert abs(np.trace(H[i]) - scale * np.sum(A[i].astype(np.float64) ** 2)) < 1e-12
+    rows, cols = [0, 5, 2], [3, 5, 1]
+    np.testing.assert_allclose(oracle.lsq_gram_entries(A, b, scale, 1, rows, cols), H[1, rows, cols], rtol=1e-14)
+
+
 def test_lsq_optimum_matches_library_solver():
     """x* minimises sum_i ||A_i x - b_i||^2: compare with numpy's SVD-based lstsq on the stacked system."""
     A, b, _ = _problem()
