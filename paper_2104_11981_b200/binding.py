@@ -60,6 +60,8 @@ _lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
 _lib.lsq_grad_workspace_bytes.restype = _i64
 _lib.lsq_grad.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp, _i64, _vp]
 _lib.lsq_grad_static.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp]
+_lib.lsq_gram_build.argtypes = [_int, _int, _int, _vp, _vp, _flt, _vp, _vp, _vp]
+_lib.lsq_grad_gram.argtypes = [_int, _int, _vp, _vp, _vp, _vp, _vp]
 _lib.dlm_launch_count.argtypes = []
 _lib.dlm_launch_count.restype = _i64
 _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
@@ -67,7 +69,7 @@ _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
            "topology_tables_device", "topology_destroy", "decentlam_step", "decentlam_step_host_gradients", "dmsgd_step", "dsgd_step", "pmsgd_step",
-           "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
+           "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "lsq_gram_build", "lsq_grad_gram", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
 def _check(rc, where):
@@ -258,6 +260,24 @@ def lsq_grad_static(A, b, x, g, scale, stream=None):
     assert b.shape == (n, p) and x.shape == (n, q) and g.shape == (n, q)
     _check(_lib.lsq_grad_static(n, p, q, _vp(A.data_ptr()), _vp(b.data_ptr()), _vp(x.data_ptr()),
                                 _vp(g.data_ptr()), scale, _stream_ptr(stream)), "lsq_grad_static")
+
+
+def lsq_gram_build(A, b, scale, H, c, stream=None):
+    """H <- scale * A_i^T A_i [n,q,q], c <- scale * A_i^T b_i [n,q] (contiguous fp32 device tensors)."""
+    n, p, q = A.shape
+    assert A.is_contiguous() and b.is_contiguous() and H.is_contiguous() and c.is_contiguous()
+    assert b.shape == (n, p) and H.shape == (n, q, q) and c.shape == (n, q)
+    _check(_lib.lsq_gram_build(n, p, q, _vp(A.data_ptr()), _vp(b.data_ptr()), scale, _vp(H.data_ptr()),
+                               _vp(c.data_ptr()), _stream_ptr(stream)), "lsq_gram_build")
+
+
+def lsq_grad_gram(H, c, x, g, stream=None):
+    """g <- H_i x_i - c_i with H, c from lsq_gram_build; x, g [n,q] contiguous fp32 device tensors."""
+    n, q, _ = H.shape
+    assert H.is_contiguous() and c.is_contiguous() and x.is_contiguous() and g.is_contiguous()
+    assert H.shape == (n, q, q) and c.shape == (n, q) and x.shape == (n, q) and g.shape == (n, q)
+    _check(_lib.lsq_grad_gram(n, q, _vp(H.data_ptr()), _vp(c.data_ptr()), _vp(x.data_ptr()), _vp(g.data_ptr()),
+                              _stream_ptr(stream)), "lsq_grad_gram")
 
 
 def launch_count():

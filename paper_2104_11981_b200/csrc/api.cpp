@@ -234,6 +234,30 @@ int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x
     return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, reinterpret_cast<float*>(workspace), cuda_stream);
 }
 
+int lsq_gram_build(int n, int p, int q, const float* A, const float* b, float scale, float* H, float* c,
+                   void* cuda_stream) {
+    if (!A || !b || !H || !c) return DLM_ERR_NULL;
+    if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
+    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if ((uintptr_t)A % 16 || (uintptr_t)H % 16 || (uintptr_t)b % 4 || (uintptr_t)c % 4) return DLM_ERR_ALIGN;
+    Range ra = span(A, n, (int64_t)p * q, (int64_t)p * q, 4), rb = span(b, n, p, p, 4),
+          rh = span(H, n, (int64_t)q * q, (int64_t)q * q, 4), rc = span(c, n, q, q, 4);
+    if (overlap(rh, ra) || overlap(rh, rb) || overlap(rc, ra) || overlap(rc, rb) || overlap(rh, rc))
+        return DLM_ERR_ALIAS;
+    return dlm_launch_gram_build(n, p, q, A, b, scale, H, c, cuda_stream);
+}
+
+int lsq_grad_gram(int n, int q, const float* H, const float* c, const float* x, float* g, void* cuda_stream) {
+    if (!H || !c || !x || !g) return DLM_ERR_NULL;
+    if (n < 1 || q < 1) return DLM_ERR_SHAPE;
+    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if ((uintptr_t)H % 16 || (uintptr_t)x % 16 || (uintptr_t)c % 4 || (uintptr_t)g % 4) return DLM_ERR_ALIGN;
+    Range rh = span(H, n, (int64_t)q * q, (int64_t)q * q, 4), rc = span(c, n, q, q, 4), rx = span(x, n, q, q, 4),
+          rg = span(g, n, q, q, 4);
+    if (overlap(rg, rh) || overlap(rg, rc) || overlap(rg, rx)) return DLM_ERR_ALIAS;
+    return dlm_launch_gram_grad(n, q, H, c, x, g, cuda_stream);
+}
+
 int64_t dlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

@@ -60,5 +60,8 @@ int dlm_launch_pmsgd(int n, int64_t d, int64_t ld, float* x, float* m, const voi
 int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
                         float scale, float* partial, void* stream);
 int dlm_lsq_splits(int n, int p, int q);  // row chunks per node used by lsq_grad
+int dlm_launch_gram_build(int n, int p, int q, const float* A, const float* b, float scale, float* H, float* c,
+                          void* stream);
+int dlm_launch_gram_grad(int n, int q, const float* H, const float* c, const float* x, float* g, void* stream);
 
 void dlm_count_launch(int launches);

@@ -433,3 +433,341 @@ extern "C" DLM_API int lsq_grad_static(int n, int p, int q, const float* A, cons
     // call, so nothing left over from an earlier call is ever consumed and nothing needs clearing.
     return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, scratch, cuda_stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Gram form of the same gradient (App. G objective expanded): A^T (A x - b) = (A^T A) x - A^T b.
+// lsq_gram_build forms H_i = scale A_i^T A_i [q, q] and c_i = scale A_i^T b_i once; afterwards every
+// gradient is the batched matrix-vector product g_i = H_i x_i - c_i, which streams n q^2 instead
+// of n p q floats.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kGramTile = 128;  // edge of the output tile of one CTA
+constexpr int kGramSlab = 8;    // rows of A per shared-memory slab
+
+template <bool VEC>
+__device__ __forceinline__ float4 gram_ld4(const float* row, int c, int q) {
+    if (VEC) {  // q % 4 == 0 and c % 4 == 0: the group is inside the row or wholly outside
+        if (c < q) return *reinterpret_cast<const float4*>(row + c);
+        return make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 v;
+    v.x = c + 0 < q ? row[c + 0] : 0.f;
+    v.y = c + 1 < q ? row[c + 1] : 0.f;
+    v.z = c + 2 < q ? row[c + 2] : 0.f;
+    v.w = c + 3 < q ? row[c + 3] : 0.f;
+    return v;
+}
+
+template <bool VEC>
+__device__ __forceinline__ void gram_st4(float* row, int c, int q, float a, float b, float cc, float d) {
+    if (VEC) {
+        if (c < q) *reinterpret_cast<float4*>(row + c) = make_float4(a, b, cc, d);
+        return;
+    }
+    if (c + 0 < q) row[c + 0] = a;
+    if (c + 1 < q) row[c + 1] = b;
+    if (c + 2 < q) row[c + 2] = cc;
+    if (c + 3 < q) row[c + 3] = d;
+}
+
+// H_i[c1, c2] = scale * sum_a A_i[a, c1] A_i[a, c2].  A CTA owns a 128 x 128 tile with c1-tile <= c2-tile
+// and writes its mirror image too, so H is bitwise symmetric; a thread owns an 8 x 8 block (two 4-wide
+// halves per direction).  Rows are summed in order with fused multiply-adds, in chunks of 256 rows:
+// each chunk's sum is scaled and added to the running value kept in H itself (read-modify-write by the
+// owning thread), which keeps the rounding error of the long sums of squares on the diagonal near
+// 1e-7 relative instead of 1e-6 for one 4096-term chain.
+constexpr int kGramChunkSlabs = 32;  // 256 rows
+
+template <bool VEC>
+__global__ void __launch_bounds__(256) gram_build_kernel(int p, int q, int tiles, float scale,
+                                                          const float* __restrict__ A, float* __restrict__ H) {
+    __shared__ __align__(16) float As[2][kGramSlab][kGramTile];  // columns of the c1 tile
+    __shared__ __align__(16) float Bs[2][kGramSlab][kGramTile];  // columns of the c2 tile
+    int t1 = 0, rem = blockIdx.x;
+    while (rem >= tiles - t1) {
+        rem -= tiles - t1;
+        ++t1;
+    }
+    const int t2 = t1 + rem;
+    const int i = blockIdx.y;
+    const float* Ai = A + (size_t)i * p * q;
+    float* Hi = H + (size_t)i * q * q;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int lr = tid >> 5, lc = (tid & 31) * 4;  // this thread's float4 of a slab
+    const int base1 = t1 * kGramTile, base2 = t2 * kGramTile;
+
+    float acc[8][8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[r][c] = 0.f;
+
+    // rows c1 = base1 + {ty*4 + r, 64 + ty*4 + r}, columns c2 = base2 + {tx*4 .., 64 + tx*4 ..}.
+    // Adds scale * acc to the running tile (or starts it) and leaves the new values in acc.
+    auto flush = [&](bool first) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int c1 = base1 + (r < 4 ? ty * 4 + r : 64 + ty * 4 + (r - 4));
+            if (c1 >= q) continue;
+            float* row = Hi + (size_t)c1 * q;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c2 = base2 + 64 * h + tx * 4;
+                float4 old = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (!first) old = gram_ld4<VEC>(row, c2, q);
+                acc[r][4 * h + 0] = fmaf(scale, acc[r][4 * h + 0], old.x);
+                acc[r][4 * h + 1] = fmaf(scale, acc[r][4 * h + 1], old.y);
+                acc[r][4 * h + 2] = fmaf(scale, acc[r][4 * h + 2], old.z);
+                acc[r][4 * h + 3] = fmaf(scale, acc[r][4 * h + 3], old.w);
+                gram_st4<VEC>(row, c2, q, acc[r][4 * h + 0], acc[r][4 * h + 1], acc[r][4 * h + 2], acc[r][4 * h + 3]);
+            }
+        }
+    };
+
+    float4 va, vb;
+    auto fetch = [&](int a0) {
+        const int a = a0 + lr;
+        if (a < p) {
+            const float* row = Ai + (size_t)a * q;
+            va = gram_ld4<VEC>(row, base1 + lc, q);
+            vb = gram_ld4<VEC>(row, base2 + lc, q);
+        } else {
+            va = vb = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    fetch(0);
+    *reinterpret_cast<float4*>(&As[0][lr][lc]) = va;
+    *reinterpret_cast<float4*>(&Bs[0][lr][lc]) = vb;
+    __syncthreads();
+    int buf = 0, slabs = 0;
+    bool first = true;
+    for (int a0 = 0; a0 < p; a0 += kGramSlab, buf ^= 1) {
+        const bool more = a0 + kGramSlab < p;
+        if (more) fetch(a0 + kGramSlab);  // in flight during the arithmetic below
+#pragma unroll
+        for (int k = 0; k < kGramSlab; ++k) {
+            const float4 a_lo = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
+            const float4 a_hi = *reinterpret_cast<const float4*>(&As[buf][k][64 + ty * 4]);
+            const float4 b_lo = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+            const float4 b_hi = *reinterpret_cast<const float4*>(&Bs[buf][k][64 + tx * 4]);
+            const float av[8] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w, a_hi.x, a_hi.y, a_hi.z, a_hi.w};
+            const float bv[8] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w, b_hi.x, b_hi.y, b_hi.z, b_hi.w};
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[r][c] = fmaf(av[r], bv[c], acc[r][c]);
+        }
+        if (more) {
+            *reinterpret_cast<float4*>(&As[buf ^ 1][lr][lc]) = va;
+            *reinterpret_cast<float4*>(&Bs[buf ^ 1][lr][lc]) = vb;
+            if (++slabs == kGramChunkSlabs) {  // a chunk is complete and more rows follow
+                flush(first);
+                first = false;
+                slabs = 0;
+#pragma unroll
+                for (int r = 0; r < 8; ++r)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) acc[r][c] = 0.f;
+            }
+        }
+        __syncthreads();
+    }
+    flush(first);  // acc now holds the final values of the tile
+    if (t1 != t2) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int c2 = base2 + (c < 4 ? tx * 4 + c : 64 + tx * 4 + (c - 4));
+            if (c2 >= q) continue;
+            float* row = Hi + (size_t)c2 * q;
+            gram_st4<VEC>(row, base1 + ty * 4, q, acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+            gram_st4<VEC>(row, base1 + 64 + ty * 4, q, acc[4][c], acc[5][c], acc[6][c], acc[7][c]);
+        }
+    }
+}
+
+// c_i[col] = scale * sum_a A_i[a, col] b_i[a].  A CTA owns 32 columns of one node; warp w takes the rows
+// a = w (mod 8) and the eight sums are added in warp order.
+__global__ void __launch_bounds__(256) gram_rhs_kernel(int p, int q, float scale, const float* __restrict__ A,
+                                                        const float* __restrict__ b, float* __restrict__ c) {
+    __shared__ float part[8][32];
+    const int i = blockIdx.y;
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int col = blockIdx.x * 32 + lane;
+    const float* Ai = A + (size_t)i * p * q;
+    const float* bi = b + (size_t)i * p;
+    float s = 0.f;
+    if (col < q) {
+        int a = grp;
+        for (; a + 24 < p; a += 32) {  // four independent loads per pass
+            const float v0 = Ai[(size_t)a * q + col], v1 = Ai[(size_t)(a + 8) * q + col];
+            const float v2 = Ai[(size_t)(a + 16) * q + col], v3 = Ai[(size_t)(a + 24) * q + col];
+            s = fmaf(v0, bi[a], s);
+            s = fmaf(v1, bi[a + 8], s);
+            s = fmaf(v2, bi[a + 16], s);
+            s = fmaf(v3, bi[a + 24], s);
+        }
+        for (; a < p; a += 8) s = fmaf(Ai[(size_t)a * q + col], bi[a], s);
+    }
+    part[grp][lane] = s;
+    __syncthreads();
+    if (grp == 0 && col < q) {
+        float v = part[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) v += part[w][lane];
+        c[(size_t)i * q + col] = scale * v;
+    }
+}
+
+// g_i[r] = <H_i[r, :], x_i> - c_i[r] for q == 128 * Q4.  Rows of H_i arrive in chunks of 8 (contiguous
+// in memory) through the same bulk-copy pipeline as lsq_partial_bulk_kernel; warp w takes row w of
+// each chunk: per-lane fused multiply-adds over the lane's float4 groups, then a butterfly sum.
+template <int Q4>
+__global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int rows_per_split,
+                                                                   const float* __restrict__ H,
+                                                                   const float* __restrict__ cvec,
+                                                                   const float* __restrict__ x,
+                                                                   float* __restrict__ g) {
+    extern __shared__ __align__(16) unsigned char lsq_smem[];
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // x may come from the kernel before this one
+    unsigned char* base = lsq_smem + ((128u - (lsq_smem_u32(lsq_smem) & 127u)) & 127u);
+    const uint32_t chunk_bytes = (uint32_t)kWarps * q * 4;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)kStages * chunk_bytes);
+    const int s = blockIdx.x, i = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = s * rows_per_split, r1 = min(q, r0 + rows_per_split);
+    const float* Hi = H + (size_t)i * q * q;
+    const float4* xi = reinterpret_cast<const float4*>(x + (size_t)i * q);
+    const float* ci = cvec + (size_t)i * q;
+    float* gi = g + (size_t)i * q;
+    const int chunks = (r1 - r0 + kWarps - 1) / kWarps;
+
+    auto issue = [&](int st, int c) {
+        const int row = r0 + c * kWarps;
+        const uint32_t bytes = (uint32_t)min(kWarps, r1 - row) * q * 4;
+        const uint32_t bar = lsq_smem_u32(&bars[st]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(lsq_smem_u32(base + (size_t)st * chunk_bytes)), "l"(Hi + (size_t)row * q), "r"(bytes), "r"(bar)
+                     : "memory");
+    };
+    if (threadIdx.x == 0) {
+        for (int st = 0; st < kStages; ++st)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lsq_smem_u32(&bars[st])), "r"(1));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int st = 0; st < kStages && st < chunks; ++st) issue(st, st);
+    }
+    float4 xr[Q4];
+#pragma unroll
+    for (int t = 0; t < Q4; ++t) xr[t] = xi[lane + 32 * t];
+    __syncthreads();
+    for (int c = 0; c < chunks; ++c) {
+        const int st = c % kStages;
+        const int r = r0 + c * kWarps + warp;
+        const float cv = r < r1 ? ci[r] : 0.f;  // in flight while the chunk lands
+        const bool arrived = lsq_mbar_wait(lsq_smem_u32(&bars[st]), (uint32_t)((c / kStages) & 1));
+        if (!__syncthreads_and(arrived)) {
+            if (threadIdx.x == 0) {
+                atomicExch(&g_lsq_kernel_error, 3);
+                for (int j = c + 1; j < chunks && j < c + kStages; ++j)
+                    lsq_mbar_wait(lsq_smem_u32(&bars[j % kStages]), (uint32_t)((j / kStages) & 1));
+            }
+            __syncthreads();
+            return;
+        }
+        if (r < r1) {
+            const float4* row = reinterpret_cast<const float4*>(base + (size_t)st * chunk_bytes) + (size_t)warp * (q >> 2);
+            float dot = 0.f;
+#pragma unroll
+            for (int t = 0; t < Q4; ++t) {
+                const float4 h = row[lane + 32 * t];
+                dot = fmaf(h.x, xr[t].x, dot);
+                dot = fmaf(h.y, xr[t].y, dot);
+                dot = fmaf(h.z, xr[t].z, dot);
+                dot = fmaf(h.w, xr[t].w, dot);
+            }
+            dot = warp_allsum(dot);
+            if (lane == 0) gi[r] = dot - cv;
+        }
+        if (c + kStages < chunks) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();  // every warp has finished reading this stage
+            if (threadIdx.x == 0) issue(st, c + kStages);
+        }
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Any q: one warp per row of H, scalar loads.
+__global__ void __launch_bounds__(kThreads) gram_grad_generic_kernel(int n, int q, const float* __restrict__ H,
+                                                                      const float* __restrict__ cvec,
+                                                                      const float* __restrict__ x,
+                                                                      float* __restrict__ g) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const long long row = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= (long long)n * q) return;
+    const int i = (int)(row / q);
+    const float* h = H + (size_t)row * q;
+    const float* xi = x + (size_t)i * q;
+    float dot = 0.f;
+    for (int c = lane; c < q; c += 32) dot = fmaf(h[c], xi[c], dot);
+    dot = warp_allsum(dot);
+    if (lane == 0) g[row] = dot - cvec[row];
+}
+
+}  // namespace
+
+int dlm_launch_gram_build(int n, int p, int q, const float* A, const float* b, float scale, float* H, float* c,
+                          void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int tiles = (q + kGramTile - 1) / kGramTile;
+    dim3 grid((unsigned)(tiles * (tiles + 1) / 2), (unsigned)n);
+    if (q % 4 == 0)
+        gram_build_kernel<true><<<grid, 256, 0, st>>>(p, q, tiles, scale, A, H);
+    else
+        gram_build_kernel<false><<<grid, 256, 0, st>>>(p, q, tiles, scale, A, H);
+    if (cudaGetLastError() != cudaSuccess) return DLM_ERR_CUDA;
+    gram_rhs_kernel<<<dim3((unsigned)((q + 31) / 32), (unsigned)n), 256, 0, st>>>(p, q, scale, A, b, c);
+    dlm_count_launch(2);
+    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
+
+int dlm_launch_gram_grad(int n, int q, const float* H, const float* c, const float* x, float* g, void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err = cudaSuccess;
+    if (q % 128 == 0 && q <= 1024) {
+        const int S = dlm_lsq_splits(n, q, q);  // row chunks per node: one wave of CTAs
+        if (S < 1) return DLM_ERR_CUDA;
+        const int rows = ((q + S - 1) / S + kWarps - 1) / kWarps * kWarps;
+        cfg.gridDim = dim3((unsigned)((q + rows - 1) / rows), (unsigned)n);
+        cfg.dynamicSmemBytes = (size_t)kStages * kWarps * q * 4 + kStages * 8 + 128 + 16;
+#define DLM_GRAM_BULK(Q4)                                                                                        \
+    case Q4: {                                                                                                   \
+        auto kern = gram_grad_bulk_kernel<Q4>;                                                                   \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg.dynamicSmemBytes) != \
+            cudaSuccess)                                                                                         \
+            return DLM_ERR_CUDA;                                                                                 \
+        err = cudaLaunchKernelEx(&cfg, kern, q, rows, H, c, x, g);                                               \
+    } break;
+        switch (q / 128) {
+            DLM_GRAM_BULK(1) DLM_GRAM_BULK(2) DLM_GRAM_BULK(3) DLM_GRAM_BULK(4)
+            DLM_GRAM_BULK(5) DLM_GRAM_BULK(6) DLM_GRAM_BULK(7) DLM_GRAM_BULK(8)
+        }
+#undef DLM_GRAM_BULK
+    } else {
+        cfg.gridDim = dim3((unsigned)(((long long)n * q + kWarps - 1) / kWarps));
+        cfg.dynamicSmemBytes = 0;
+        err = cudaLaunchKernelEx(&cfg, gram_grad_generic_kernel, n, q, H, c, x, g);
+    }
+    dlm_count_launch(1);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
