@@ -224,3 +224,44 @@ def test_lsq_argument_validation_on_host():
     assert lib.lsq_grad_workspace_bytes(0, 1, 1) == -2 and lib.lsq_grad_workspace_bytes(1, 1, 9000) == -8
     with pytest.raises(B.DecentlamError):
         B.lsq_grad_workspace_bytes(1, 0, 1)
+
+
+def test_gram_argument_validation_on_host():
+    lib = B.raw()
+    vp = ctypes.c_void_p
+    A, Bv, Hm, Cv, X, G, M, Xo = (0x10000000, 0x50000000, 0x60000000, 0x90000000, 0xA0000000, 0xB0000000, 0xC0000000,
+                                  0xD0000000)
+    n, p, q = 4, 64, 128
+
+    def build(**kw):
+        return lib.lsq_gram_build(kw.get("n", n), kw.get("p", p), kw.get("q", q), vp(kw.get("A", A)), vp(kw.get("b", Bv)),
+                                  1.0 / p, vp(kw.get("H", Hm)), vp(kw.get("c", Cv)), None)
+
+    assert build(A=0) == -1 and build(H=0) == -1 and build(c=0) == -1
+    assert build(n=0) == -2 and build(p=0) == -2 and build(q=8193) == -8
+    assert build(A=A + 4) == -3 and build(H=Hm + 8) == -3
+    assert build(H=A) == -4 and build(c=Bv) == -4 and build(c=Hm) == -4
+
+    def grad(**kw):
+        return lib.lsq_grad_gram(kw.get("n", n), kw.get("q", q), vp(kw.get("H", Hm)), vp(kw.get("c", Cv)),
+                                 vp(kw.get("x", X)), vp(kw.get("g", G)), None)
+
+    assert grad(H=0) == -1 and grad(g=0) == -1
+    assert grad(n=0) == -2 and grad(q=0) == -2 and grad(q=8193) == -8
+    assert grad(x=X + 4) == -3 and grad(H=Hm + 4) == -3
+    assert grad(g=X) == -4 and grad(g=Cv) == -4 and grad(g=Hm) == -4
+
+    topo = B.topology_build(B.RING, n)
+
+    def step(**kw):
+        return lib.lsq_gram_step(kw.get("rule", 0), kw.get("topo", topo.handle), kw.get("k", 0), kw.get("n", n),
+                                 kw.get("q", q), vp(kw.get("H", Hm)), vp(kw.get("c", Cv)), vp(kw.get("x", X)),
+                                 vp(kw.get("m", M)), vp(kw.get("xo", Xo)), kw.get("beta", 0.9), kw.get("gamma", 0.1), None)
+
+    assert step(rule=3) == -6
+    assert step(H=0) == -1 and step(xo=0) == -1 and step(topo=None) == -1
+    assert step(n=0) == -2 and step(k=-1) == -2 and step(n=5) == -2     # n differs from the topology's
+    assert step(q=100) == -8 and step(q=1152) == -8
+    assert step(x=X + 4) == -3
+    assert step(gamma=0.0) == -5 and step(beta=1.0) == -5
+    assert step(xo=X) == -4 and step(xo=M) == -4 and step(m=X) == -4 and step(xo=Cv) == -4
