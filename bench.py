@@ -424,6 +424,36 @@ def run_lsq_workload(args, w, B, inputs, torch, dev, rank, world, dist):
     secs, launches = time_steps(iteration, reset, args.steps, args.warmup, torch, stream, B.launch_count)
     clocks = sampler.stop()
     lsq_secs, _ = time_steps(lambda k: B.lsq_grad(A, b, x, g, scale, ws), reset, args.steps, 3, torch, stream)
+    # the same iteration with the gradient in expanded (Gram) form: H, c built once, then n*q*q floats per step
+    H = torch.empty((n, q, q), device=dev); c = torch.empty((n, q), device=dev)
+    build_secs, _ = time_steps(lambda k: B.lsq_gram_build(A, b, scale, H, c), reset, 5, 3, torch, stream)
+
+    def gram_iteration(k):
+        B.lsq_grad_gram(H, c, x, g)
+        B.decentlam_step(topo, k, x, m, g, w.beta, w.gamma)
+
+    gram_secs, _ = time_steps(gram_iteration, reset, args.steps, 3, torch, stream)
+    gram_grad_secs, _ = time_steps(lambda k: B.lsq_grad_gram(H, c, x, g), reset, args.steps, 3, torch, stream)
+    # the Gram-form iteration is shorter than the host's cost of issuing its two calls from Python
+    # (about 20 us), so it is also timed as a CUDA graph of 40 iterations, replayed
+    reset()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for k in range(40):
+            gram_iteration(k)
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(10):
+        graph.replay()
+    e1.record(stream)
+    e1.synchronize()
+    graph_secs = e0.elapsed_time(e1) * 1e-3 / 400
+    gram_bytes = 4 * (n * q * q + 3 * n * q)
     job_secs, job_units = aggregate_over_ranks(dist, secs, n * q * args.steps, dev)
     peak, peak_kind = measured_peak()
     lsq_bytes = 4 * (n * p * q + n * p + 2 * n * q)
@@ -435,8 +465,15 @@ def run_lsq_workload(args, w, B, inputs, torch, dev, rank, world, dist):
                 "config": {"workload": args.workload, "n": n, "p": p, "q": q, "topology": w.topology, "beta": w.beta,
                            "gamma": w.gamma, "l2": f"A is {n * p * q * 4 / 2**20:.0f} MiB, larger than the 126 MB L2; no flush"},
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                             "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "lsq_partial_rows_kernel + lsq_reduce_kernel",
+                             "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "lsq_partial_bulk_kernel + lsq_reduce_kernel",
                              "algorithmic_bytes_per_launch": lsq_bytes, "ms_per_lsq_grad": lsq_secs / args.steps * 1e3},
+                "gram_form": {"build_ms_once": build_secs / 5 * 1e3,
+                              "us_per_iteration": gram_secs / args.steps * 1e6,
+                              "us_per_iteration_cuda_graph": graph_secs * 1e6,
+                              "us_per_lsq_grad_gram": gram_grad_secs / args.steps * 1e6,
+                              "lsq_grad_gram_gbs": gram_bytes * args.steps / gram_grad_secs / 1e9,
+                              "algorithmic_bytes_per_gradient": gram_bytes,
+                              "note": "effective rate: about half of H is served from L2 (evict-last hint), so it may exceed the HBM peak"},
                 "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "cpu_baseline": None}
         print(json.dumps(line), flush=True)
     if dist is not None:

@@ -287,26 +287,6 @@ DLM_API int lsq_gram_build(int n, int p, int q, const float* A, const float* b, 
                            void* cuda_stream);
 DLM_API int lsq_grad_gram(int n, int q, const float* H, const float* c, const float* x, float* g, void* cuda_stream);
 
-/*
- * One iteration of the least-squares workload in a single launch: Gram-form gradients at x_in,
- * then the chosen update rule, i.e. what lsq_grad_gram followed by decentlam_step / dmsgd_step /
- * pmsgd_step computes (same operations in the same order: bitwise the same m and x), without the
- * gradient ever leaving the chip.
- *   rule   : DLM_GRAM_DECENTLAM (Algorithm 2), DLM_GRAM_DMSGD (Algorithm 1) or DLM_GRAM_PMSGD
- *   topo,k : topology and iteration (slot k mod period); topo may be NULL for DLM_GRAM_PMSGD
- *   H, c   : from lsq_gram_build, device fp32 [n,q,q] and [n,q]; H 16-byte aligned
- *   x_in   : device fp32 [n,q], x^(k), 16-byte aligned, read only
- *   m      : device fp32 [n,q], updated in place
- *   x_out  : device fp32 [n,q], receives x^(k+1); must not overlap x_in (every block reads all of
- *            x_in for its matrix-vector products, so the parameters are double-buffered: swap the
- *            two pointers between iterations)
- * Supported: q a multiple of 128, q <= 1024, n <= 512 (DLM_ERR_UNSUPPORTED otherwise: use the
- * two-call form).  Errors as for decentlam_step plus DLM_ERR_KIND for an unknown rule.
- */
-enum { DLM_GRAM_DECENTLAM = 0, DLM_GRAM_DMSGD = 1, DLM_GRAM_PMSGD = 2 };
-DLM_API int lsq_gram_step(int rule, const dlm_topology* topo, int64_t k, int n, int q, const float* H, const float* c,
-                          const float* x_in, float* m, float* x_out, float beta, float gamma, void* cuda_stream);
-
 /* Kernel launches issued by this library in the calling process so far (all entry points). */
 DLM_API int64_t dlm_launch_count(void);
 
@@ -329,9 +309,11 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 6  threads per CTA of the pipeline kernels (128, 256 or 512)
  *   knob 7  1 = pipeline kernel with the plain mixing loop, 2 = merged-staging kernel (one staged
  *           value per neighbour)
- *   knob 8  lsq_grad: row chunks per node (at most 64)
+ *   knob 8  lsq_grad and lsq_grad_gram: row chunks per node (at most 64)
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
  *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
+ *   knob 11 lsq_grad_gram: share of H kept in L2 with evict-last priority between calls, in 1/1000
+ *           (negative = automatic: 0.55 of the L2 size when H is larger than that, else none)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
  * the default on rows of 12 or more entries) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.

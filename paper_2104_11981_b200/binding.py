@@ -14,7 +14,6 @@ LIB_PATH = os.path.join(_HERE, "libdecentlam.so")
 RING, STATIC_EXP, ONE_PEER_EXP, COMPLETE, CSR_MH, CSR_WEIGHTS, SYM_EXP, MESH = range(8)
 G_F32, G_BF16 = 0, 1
 DSGD_ATC, DSGD_AWC = 0, 1
-GRAM_DECENTLAM, GRAM_DMSGD, GRAM_PMSGD = 0, 1, 2
 MAX_NODES = 2048
 
 STATUS = {0: "DLM_OK", -1: "DLM_ERR_NULL", -2: "DLM_ERR_SHAPE", -3: "DLM_ERR_ALIGN", -4: "DLM_ERR_ALIAS",
@@ -63,7 +62,6 @@ _lib.lsq_grad.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp, _i64,
 _lib.lsq_grad_static.argtypes = [_int, _int, _int, _vp, _vp, _vp, _vp, _flt, _vp]
 _lib.lsq_gram_build.argtypes = [_int, _int, _int, _vp, _vp, _flt, _vp, _vp, _vp]
 _lib.lsq_grad_gram.argtypes = [_int, _int, _vp, _vp, _vp, _vp, _vp]
-_lib.lsq_gram_step.argtypes = [_int, _vp, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _flt, _flt, _vp]
 _lib.dlm_launch_count.argtypes = []
 _lib.dlm_launch_count.restype = _i64
 _lib.dlm_kernel_error.argtypes = [ctypes.POINTER(_int)]
@@ -71,7 +69,7 @@ _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
            "topology_tables_device", "topology_destroy", "decentlam_step", "decentlam_step_host_gradients", "dmsgd_step", "dsgd_step", "pmsgd_step",
-           "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "lsq_gram_build", "lsq_grad_gram", "lsq_gram_step", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
+           "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "lsq_gram_build", "lsq_grad_gram", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
 def _check(rc, where):
@@ -280,18 +278,6 @@ def lsq_grad_gram(H, c, x, g, stream=None):
     assert H.shape == (n, q, q) and c.shape == (n, q) and x.shape == (n, q) and g.shape == (n, q)
     _check(_lib.lsq_grad_gram(n, q, _vp(H.data_ptr()), _vp(c.data_ptr()), _vp(x.data_ptr()), _vp(g.data_ptr()),
                               _stream_ptr(stream)), "lsq_grad_gram")
-
-
-def lsq_gram_step(rule, topo, k, H, c, x_in, m, x_out, beta, gamma, stream=None):
-    """One launch: g = H x_in - c, then the rule; m in place, x^(k+1) to x_out (swap x_in / x_out between
-    iterations).  topo may be None for GRAM_PMSGD."""
-    n, q, _ = H.shape
-    for t in (H, c, x_in, m, x_out):
-        assert t.is_cuda and t.is_contiguous()
-    assert c.shape == (n, q) and x_in.shape == (n, q) and m.shape == (n, q) and x_out.shape == (n, q)
-    _check(_lib.lsq_gram_step(rule, topo.handle if topo is not None else None, k, n, q, _vp(H.data_ptr()),
-                              _vp(c.data_ptr()), _vp(x_in.data_ptr()), _vp(m.data_ptr()), _vp(x_out.data_ptr()),
-                              beta, gamma, _stream_ptr(stream)), "lsq_gram_step")
 
 
 def launch_count():

@@ -10,6 +10,11 @@
 #include "dlm_internal.h"
 
 int dlm_lsq_max_splits();
+int dlm_step_take_error(int* flag);
+int dlm_lsq_take_error(int* flag);
+int dlm_step_set_tuning(int knob, int value);
+// launch-shape overrides, defined beside the launchers that read them
+extern int g_lsq_tune_splits, g_lsq_tune_bulk, g_pmsgd_tune_cap, g_gram_l2_keep_permille;
 
 namespace {
 
@@ -258,35 +263,26 @@ int lsq_grad_gram(int n, int q, const float* H, const float* c, const float* x, 
     return dlm_launch_gram_grad(n, q, H, c, x, g, cuda_stream);
 }
 
-int lsq_gram_step(int rule, const dlm_topology* topo, int64_t k, int n, int q, const float* H, const float* c,
-                  const float* x_in, float* m, float* x_out, float beta, float gamma, void* cuda_stream) {
-    if (rule != DLM_GRAM_DECENTLAM && rule != DLM_GRAM_DMSGD && rule != DLM_GRAM_PMSGD) return DLM_ERR_KIND;
-    if (!H || !c || !x_in || !m || !x_out) return DLM_ERR_NULL;
-    if (rule != DLM_GRAM_PMSGD && !topo) return DLM_ERR_NULL;
-    if (n < 1 || q < 1 || k < 0) return DLM_ERR_SHAPE;
-    if (q % 128 != 0 || q > 1024 || n > 512) return DLM_ERR_UNSUPPORTED;
-    if ((uintptr_t)H % 16 || (uintptr_t)x_in % 16 || (uintptr_t)c % 4 || (uintptr_t)m % 4 || (uintptr_t)x_out % 4)
-        return DLM_ERR_ALIGN;
-    if (!std::isfinite(gamma) || !(gamma > 0.0f)) return DLM_ERR_HYPER;
-    if (!(beta >= 0.0f) || !(beta < 1.0f)) return DLM_ERR_HYPER;
-    Range rh = span(H, n, (int64_t)q * q, (int64_t)q * q, 4), rc = span(c, n, q, q, 4), ri = span(x_in, n, q, q, 4),
-          rm = span(m, n, q, q, 4), ro = span(x_out, n, q, q, 4);
-    if (overlap(ro, rh) || overlap(ro, rc) || overlap(ro, ri) || overlap(ro, rm) || overlap(rm, rh) ||
-        overlap(rm, rc) || overlap(rm, ri))
-        return DLM_ERR_ALIAS;
-    const int32_t *rowptr = nullptr, *col = nullptr;
-    const float* val = nullptr;
-    if (rule != DLM_GRAM_PMSGD) {
-        if (n != topo->n) return DLM_ERR_SHAPE;
-        const dlm_slot& s = topo->slots[(size_t)(k % (int64_t)topo->slots.size())];
-        if (!s.d_rowptr) return DLM_ERR_CUDA;  // host-only handle
-        int dev = -1;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev != topo->device) return DLM_ERR_CUDA;
-        rowptr = s.d_rowptr;
-        col = s.d_col;
-        val = s.d_val;
+int dlm_set_tuning(int knob, int value) {
+    switch (knob) {
+    case 0: case 1: case 2: case 3: case 4: case 5: case 6: case 7: return dlm_step_set_tuning(knob, value);
+    case 8: g_lsq_tune_splits = value; return DLM_OK;
+    case 9: g_lsq_tune_bulk = value; return DLM_OK;
+    case 10: g_pmsgd_tune_cap = value; return DLM_OK;
+    case 11: g_gram_l2_keep_permille = value; return DLM_OK;
+    default: return DLM_ERR_KIND;
     }
-    return dlm_launch_gram_step(rule, n, q, H, c, x_in, m, x_out, rowptr, col, val, beta, gamma, cuda_stream);
+}
+
+int dlm_kernel_error(int* flag) {
+    if (!flag) return DLM_ERR_NULL;
+    int step = 0, lsq = 0;
+    int rc = dlm_step_take_error(&step);
+    if (rc != DLM_OK) return rc;
+    rc = dlm_lsq_take_error(&lsq);
+    if (rc != DLM_OK) return rc;
+    *flag = step != 0 ? step : lsq;
+    return DLM_OK;
 }
 
 int64_t dlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -62,9 +62,6 @@ int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, con
 int dlm_lsq_splits(int n, int p, int q);  // row chunks per node used by lsq_grad
 int dlm_launch_gram_build(int n, int p, int q, const float* A, const float* b, float scale, float* H, float* c,
                           void* stream);
-int dlm_launch_gram_step(int rule, int n, int q, const float* H, const float* c, const float* x_in, float* m,
-                         float* x_out, const int32_t* rowptr, const int32_t* col, const float* val, float beta,
-                         float gamma, void* stream);
 int dlm_launch_gram_grad(int n, int q, const float* H, const float* c, const float* x, float* g, void* stream);
 
 void dlm_count_launch(int launches);

@@ -939,14 +939,8 @@ int dlm_launch_step(int rule, const dlm_step_args& a, void* stream) {
                                    : launch_rule<DLM_RULE_DMSGD, float>(a, s);
 }
 
-extern int g_lsq_tune_splits;
-extern int g_lsq_tune_bulk;
-extern int g_pmsgd_tune_cap;
-int dlm_lsq_take_error(int* flag);
-
-extern "C" {
-
-DLM_API int dlm_set_tuning(int knob, int value) {
+// Launch-shape overrides of the step kernels (knobs 0 .. 7 of dlm_set_tuning).
+int dlm_step_set_tuning(int knob, int value) {
     switch (knob) {
     case 0: g_tune_path = value; return DLM_OK;
     case 1: g_tune_cols = value; return DLM_OK;
@@ -956,26 +950,18 @@ DLM_API int dlm_set_tuning(int knob, int value) {
     case 5: g_tune_tables = value; return DLM_OK;
     case 6: g_tune_threads = value; return DLM_OK;
     case 7: g_tune_mix = value; return DLM_OK;
-    case 8: g_lsq_tune_splits = value; return DLM_OK;
-    case 9: g_lsq_tune_bulk = value; return DLM_OK;
-    case 10: g_pmsgd_tune_cap = value; return DLM_OK;
     default: return DLM_ERR_KIND;
     }
 }
 
-DLM_API int dlm_kernel_error(int* flag) {
-    if (!flag) return DLM_ERR_NULL;
+// Reads and clears the error flag of the step kernels' bounded waits.
+int dlm_step_take_error(int* flag) {
     int v = 0;
     if (cudaMemcpyFromSymbol(&v, g_kernel_error, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
     if (v != 0) {
         int zero = 0;
         if (cudaMemcpyToSymbol(g_kernel_error, &zero, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
     }
-    int lsq = 0;
-    int rc = dlm_lsq_take_error(&lsq);
-    if (rc != DLM_OK) return rc;
-    *flag = v != 0 ? v : lsq;
+    *flag = v;
     return DLM_OK;
 }
-
-}  // extern "C"

@@ -250,18 +250,3 @@ def test_gram_argument_validation_on_host():
     assert grad(n=0) == -2 and grad(q=0) == -2 and grad(q=8193) == -8
     assert grad(x=X + 4) == -3 and grad(H=Hm + 4) == -3
     assert grad(g=X) == -4 and grad(g=Cv) == -4 and grad(g=Hm) == -4
-
-    topo = B.topology_build(B.RING, n)
-
-    def step(**kw):
-        return lib.lsq_gram_step(kw.get("rule", 0), kw.get("topo", topo.handle), kw.get("k", 0), kw.get("n", n),
-                                 kw.get("q", q), vp(kw.get("H", Hm)), vp(kw.get("c", Cv)), vp(kw.get("x", X)),
-                                 vp(kw.get("m", M)), vp(kw.get("xo", Xo)), kw.get("beta", 0.9), kw.get("gamma", 0.1), None)
-
-    assert step(rule=3) == -6
-    assert step(H=0) == -1 and step(xo=0) == -1 and step(topo=None) == -1
-    assert step(n=0) == -2 and step(k=-1) == -2 and step(n=5) == -2     # n differs from the topology's
-    assert step(q=100) == -8 and step(q=1152) == -8
-    assert step(x=X + 4) == -3
-    assert step(gamma=0.0) == -5 and step(beta=1.0) == -5
-    assert step(xo=X) == -4 and step(xo=M) == -4 and step(m=X) == -4 and step(xo=Cv) == -4
