@@ -51,10 +51,10 @@ def parse_args():
 # SHA-256 matches, otherwise "traffic" is null.
 NCU_CAPTURE = {
     "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
-    "sha256": "78aebba5a62c2a2883cd13650a01f28f2180faf09af264398e8e503666a977c9",
+    "sha256": "ec754a260b423fe21ac4b8ac812bea14992768a991f78dbd234a551fc11f6982",
     "workload": "cfg2",
-    "dram_read_bytes_per_np": 402.69e6 / (16 * 2097152),
-    "dram_write_bytes_per_np": 214.79e6 / (16 * 2097152),
+    "dram_read_bytes_per_np": 402.70e6 / (16 * 2097152),
+    "dram_write_bytes_per_np": 211.67e6 / (16 * 2097152),
 }
 
 
