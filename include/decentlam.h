@@ -313,7 +313,8 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
  *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
  *   knob 11 lsq_grad_gram: share of H kept in L2 with evict-last priority between calls, in 1/1000
- *           (negative = automatic: 0.55 of the L2 size when H is larger than that, else none)
+ *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
+ *           size, else none)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
  * the default on rows of 12 or more entries) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.

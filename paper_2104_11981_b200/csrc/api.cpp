@@ -14,7 +14,7 @@ int dlm_step_take_error(int* flag);
 int dlm_lsq_take_error(int* flag);
 int dlm_step_set_tuning(int knob, int value);
 // launch-shape overrides, defined beside the launchers that read them
-extern int g_lsq_tune_splits, g_lsq_tune_bulk, g_pmsgd_tune_cap, g_gram_l2_keep_permille;
+extern int g_lsq_tune_splits, g_lsq_tune_bulk, g_pmsgd_tune_cap, g_l2_keep_permille;
 
 namespace {
 
@@ -269,7 +269,7 @@ int dlm_set_tuning(int knob, int value) {
     case 8: g_lsq_tune_splits = value; return DLM_OK;
     case 9: g_lsq_tune_bulk = value; return DLM_OK;
     case 10: g_pmsgd_tune_cap = value; return DLM_OK;
-    case 11: g_gram_l2_keep_permille = value; return DLM_OK;
+    case 11: g_l2_keep_permille = value; return DLM_OK;
     default: return DLM_ERR_KIND;
     }
 }

@@ -114,6 +114,27 @@ __device__ __forceinline__ bool lsq_mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 
+// L2 policy for the bulk copies of a matrix that every iteration reads again (H of the Gram form):
+// the given fraction of its lines is kept with evict-last priority so that it is still cached at the
+// next call, the rest is marked evict-first.
+__device__ __forceinline__ uint64_t keep_policy(float keep) {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.L2::evict_first.b64 %0, %1;" : "=l"(pol) : "f"(keep));
+    return pol;
+}
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, bool hint,
+                                               uint64_t pol) {
+    if (hint)
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+            ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+            : "memory");
+    else
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                     : "memory");
+}
+
 template <int Q4>
 __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q, int rows_per_split, int splits,
                                                                      const float* __restrict__ A,
@@ -139,9 +160,7 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
         const uint32_t bytes = (uint32_t)min(kWarps, r1 - row) * q * 4;
         const uint32_t bar = lsq_smem_u32(&bars[st]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(lsq_smem_u32(base + (size_t)st * chunk_bytes)), "l"(Ai + (size_t)row * q), "r"(bytes), "r"(bar)
-                     : "memory");
+        bulk_copy(lsq_smem_u32(base + (size_t)st * chunk_bytes), Ai + (size_t)row * q, bytes, bar, false, 0);
     };
     if (threadIdx.x == 0) {
         for (int st = 0; st < kStages; ++st)
@@ -306,6 +325,23 @@ int dlm_lsq_splits(int n, int p, int q) {
     S = std::min(S, std::max(1, p / (4 * kWarps)));
     int rows = ((p + S - 1) / S + kWarps - 1) / kWarps * kWarps;
     return (p + rows - 1) / rows;
+}
+
+int g_l2_keep_permille = -1;  // share of H kept in L2 between calls, in 1/1000; < 0 = automatic
+
+// Fraction of H (`bytes` bytes) to keep in L2 with evict-last priority.  Every iteration reads all of H
+// again, and a cyclic sweep over more bytes than the cache holds evicts every line just before its
+// reuse; pinning as much as comfortably fits (0.55 of the cache measured best on a 126 MB L2) turns
+// that share of the traffic into hits.  Nothing is pinned when H fits anyway, nor when it is more
+// than twice the cache: on the 537 MB matrix of the residual form the same hint gained 0 to 6 %,
+// erratically, so it is used only where it was measured to pay.
+static float l2_keep_fraction(double bytes) {
+    if (g_l2_keep_permille >= 0) return std::min(1.0f, g_l2_keep_permille / 1000.0f);
+    int dev = 0, l2 = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
+        return 0.0f;
+    const double room = 0.55 * (double)l2;
+    return (bytes <= room || bytes > 2.0 * (double)l2) ? 0.0f : (float)(room / bytes);
 }
 
 int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
@@ -622,26 +658,6 @@ __global__ void __launch_bounds__(256) gram_rhs_kernel(int p, int q, float scale
 // g_i[r] = <H_i[r, :], x_i> - c_i[r] for q == 128 * Q4.  Rows of H_i arrive in chunks of 8 (contiguous
 // in memory) through the same bulk-copy pipeline as lsq_partial_bulk_kernel; warp w takes row w of
 // each chunk: per-lane fused multiply-adds over the lane's float4 groups, then a butterfly sum.
-// L2 policy for the copies of H: the given fraction of its lines is kept with evict-last priority so
-// that it is still cached when the next iteration reads H again, the rest is marked evict-first.
-__device__ __forceinline__ uint64_t gram_keep_policy(float keep) {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.L2::evict_first.b64 %0, %1;" : "=l"(pol) : "f"(keep));
-    return pol;
-}
-__device__ __forceinline__ void gram_bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, bool hint,
-                                               uint64_t pol) {
-    if (hint)
-        asm volatile(
-            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-            ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol)
-            : "memory");
-    else
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                     : "memory");
-}
-
 template <int Q4>
 __global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int rows_per_split, float l2_keep,
                                                                    const float* __restrict__ H,
@@ -662,14 +678,14 @@ __global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int row
     float* gi = g + (size_t)i * q;
     const int chunks = (r1 - r0 + kWarps - 1) / kWarps;
     const bool hint = l2_keep > 0.f;
-    const uint64_t pol = hint ? gram_keep_policy(l2_keep) : 0;
+    const uint64_t pol = hint ? keep_policy(l2_keep) : 0;
 
     auto issue = [&](int st, int c) {
         const int row = r0 + c * kWarps;
         const uint32_t bytes = (uint32_t)min(kWarps, r1 - row) * q * 4;
         const uint32_t bar = lsq_smem_u32(&bars[st]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        gram_bulk_copy(lsq_smem_u32(base + (size_t)st * chunk_bytes), Hi + (size_t)row * q, bytes, bar, hint, pol);
+        bulk_copy(lsq_smem_u32(base + (size_t)st * chunk_bytes), Hi + (size_t)row * q, bytes, bar, hint, pol);
     };
     if (threadIdx.x == 0) {
         for (int st = 0; st < kStages; ++st)
@@ -753,25 +769,9 @@ int dlm_launch_gram_build(int n, int p, int q, const float* A, const float* b, f
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-int g_gram_l2_keep_permille = -1;  // fraction of H kept in L2 between calls, in 1/1000; < 0 = automatic
-
-// Fraction of H [n, q, q] to keep in L2 with evict-last priority.  An iteration reads all of H again,
-// and a cyclic sweep over more bytes than the cache holds evicts every line just before its reuse;
-// pinning as much of H as comfortably fits (0.55 of the cache measured best on a 126 MB L2: 12.5
-// instead of 18.8 us per gradient at n = 32, q = 1024) turns that share of the traffic into hits.
-// Nothing is pinned when H fits anyway.
-static float gram_l2_keep(int n, int q) {
-    if (g_gram_l2_keep_permille >= 0) return std::min(1.0f, g_gram_l2_keep_permille / 1000.0f);
-    int dev = 0, l2 = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
-        return 0.0f;
-    const double bytes = (double)n * q * q * 4.0, room = 0.55 * (double)l2;
-    return bytes <= room ? 0.0f : (float)(room / bytes);
-}
-
 int dlm_launch_gram_grad(int n, int q, const float* H, const float* c, const float* x, float* g, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const float keep = gram_l2_keep(n, q);
+    const float keep = l2_keep_fraction((double)n * q * q * 4.0);
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kThreads);
     cfg.stream = st;
