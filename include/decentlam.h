@@ -215,7 +215,7 @@ DLM_API int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const v
 /* ------------------------------------------------------------------------------------
  * Full-batch least-squares gradient of the linear-regression experiment (App. G):
  *   f_i(x) = (scale/2) ||A_i x - b_i||^2 ,   g_i = scale * A_i^T (A_i x_i - b_i).
- *   A : device fp32 [n, p, q] row-major, 16-byte aligned; 1 <= q <= 8192
+ *   A : device fp32 [n, p, q] row-major, 16-byte aligned; 1 <= q <= 8192, n <= DLM_LSQ_MAX_NODES
  *   b : device fp32 [n, p];  x : device fp32 [n, q] (row stride q), 16-byte aligned;
  *   g : device fp32 [n, q], 16-byte aligned, written
  *   workspace, workspace_bytes : device scratch of at least lsq_grad_workspace_bytes(n,p,q)
@@ -225,8 +225,9 @@ DLM_API int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const v
  * kernel that re-reads each 8-row block from cache.  Partial sums are combined in a fixed
  * order, so repeated calls give bitwise identical results.
  * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_UNSUPPORTED
- *         (q above 8192), DLM_ERR_WORKSPACE, DLM_ERR_CUDA.
+ *         (q above 8192 or n above DLM_LSQ_MAX_NODES), DLM_ERR_WORKSPACE, DLM_ERR_CUDA.
  * ------------------------------------------------------------------------------------ */
+#define DLM_LSQ_MAX_NODES 65535 /* nodes are one grid dimension of the least-squares kernels */
 DLM_API int64_t lsq_grad_workspace_bytes(int n, int p, int q); /* negative dlm_status on bad sizes */
 
 DLM_API int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,

@@ -219,7 +219,7 @@ int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const void* g, 
 
 int64_t lsq_grad_workspace_bytes(int n, int p, int q) {
     if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
-    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if (q > 8192 || n > DLM_LSQ_MAX_NODES) return DLM_ERR_UNSUPPORTED;
     return (int64_t)n * dlm_lsq_max_splits() * q * 4;
 }
 
@@ -227,7 +227,7 @@ int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x
              void* workspace, int64_t workspace_bytes, void* cuda_stream) {
     if (!A || !b || !x || !g) return DLM_ERR_NULL;
     if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
-    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if (q > 8192 || n > DLM_LSQ_MAX_NODES) return DLM_ERR_UNSUPPORTED;
     if ((uintptr_t)A % 16 || (uintptr_t)x % 16 || (uintptr_t)g % 16 || (uintptr_t)b % 4) return DLM_ERR_ALIGN;
     if (!workspace || (uintptr_t)workspace % 256 || workspace_bytes < lsq_grad_workspace_bytes(n, p, q))
         return DLM_ERR_WORKSPACE;
@@ -243,7 +243,7 @@ int lsq_gram_build(int n, int p, int q, const float* A, const float* b, float sc
                    void* cuda_stream) {
     if (!A || !b || !H || !c) return DLM_ERR_NULL;
     if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
-    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if (q > 8192 || n > DLM_LSQ_MAX_NODES) return DLM_ERR_UNSUPPORTED;
     if ((uintptr_t)A % 16 || (uintptr_t)H % 16 || (uintptr_t)b % 4 || (uintptr_t)c % 4) return DLM_ERR_ALIGN;
     Range ra = span(A, n, (int64_t)p * q, (int64_t)p * q, 4), rb = span(b, n, p, p, 4),
           rh = span(H, n, (int64_t)q * q, (int64_t)q * q, 4), rc = span(c, n, q, q, 4);
@@ -255,7 +255,7 @@ int lsq_gram_build(int n, int p, int q, const float* A, const float* b, float sc
 int lsq_grad_gram(int n, int q, const float* H, const float* c, const float* x, float* g, void* cuda_stream) {
     if (!H || !c || !x || !g) return DLM_ERR_NULL;
     if (n < 1 || q < 1) return DLM_ERR_SHAPE;
-    if (q > 8192) return DLM_ERR_UNSUPPORTED;
+    if (q > 8192 || n > DLM_LSQ_MAX_NODES) return DLM_ERR_UNSUPPORTED;
     if ((uintptr_t)H % 16 || (uintptr_t)x % 16 || (uintptr_t)c % 4 || (uintptr_t)g % 4) return DLM_ERR_ALIGN;
     Range rh = span(H, n, (int64_t)q * q, (int64_t)q * q, 4), rc = span(c, n, q, q, 4), rx = span(x, n, q, q, 4),
           rg = span(g, n, q, q, 4);

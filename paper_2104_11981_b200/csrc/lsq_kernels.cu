@@ -454,7 +454,7 @@ extern "C" DLM_API int lsq_grad_static(int n, int p, int q, const float* A, cons
                                        float* g, float scale, void* cuda_stream) {
     if (!A || !b || !x || !g) return DLM_ERR_NULL;
     if (n < 1 || p < 1 || q < 1) return DLM_ERR_SHAPE;
-    if (q > kGenericMaxQ) return DLM_ERR_UNSUPPORTED;
+    if (q > kGenericMaxQ || n > DLM_LSQ_MAX_NODES) return DLM_ERR_UNSUPPORTED;
     if ((uintptr_t)A % 16 || (uintptr_t)x % 16 || (uintptr_t)g % 16 || (uintptr_t)b % 4) return DLM_ERR_ALIGN;
     const size_t ab = (size_t)n * p * q * 4, bb = (size_t)n * p * 4, xb = (size_t)n * q * 4;
     if (ranges_overlap(g, xb, A, ab) || ranges_overlap(g, xb, b, bb) || ranges_overlap(g, xb, x, xb))

@@ -217,7 +217,7 @@ def test_lsq_argument_validation_on_host():
 
     assert call(A=0) == -1 and call(g=0) == -1
     assert call(n=0) == -2 and call(q=0) == -2
-    assert call(q=8193) == -8
+    assert call(q=8193) == -8 and call(n=65536) == -8
     assert call(A=A + 4) == -3 and call(x=X + 8) == -3
     assert call(ws=0) == -10 and call(ws=Wk + 64) == -10 and call(wsb=need - 1) == -10
     assert call(g=X) == -4 and call(ws=G) == -4
@@ -238,7 +238,7 @@ def test_gram_argument_validation_on_host():
                                   1.0 / p, vp(kw.get("H", Hm)), vp(kw.get("c", Cv)), None)
 
     assert build(A=0) == -1 and build(H=0) == -1 and build(c=0) == -1
-    assert build(n=0) == -2 and build(p=0) == -2 and build(q=8193) == -8
+    assert build(n=0) == -2 and build(p=0) == -2 and build(q=8193) == -8 and build(n=65536) == -8
     assert build(A=A + 4) == -3 and build(H=Hm + 8) == -3
     assert build(H=A) == -4 and build(c=Bv) == -4 and build(c=Hm) == -4
 
@@ -247,6 +247,6 @@ def test_gram_argument_validation_on_host():
                                  vp(kw.get("x", X)), vp(kw.get("g", G)), None)
 
     assert grad(H=0) == -1 and grad(g=0) == -1
-    assert grad(n=0) == -2 and grad(q=0) == -2 and grad(q=8193) == -8
+    assert grad(n=0) == -2 and grad(q=0) == -2 and grad(q=8193) == -8 and grad(n=65536) == -8
     assert grad(x=X + 4) == -3 and grad(H=Hm + 4) == -3
     assert grad(g=X) == -4 and grad(g=Cv) == -4 and grad(g=Hm) == -4
