@@ -13,7 +13,11 @@
  *   - The step functions and lsq_grad only enqueue work on `cuda_stream` (a cudaStream_t
  *     cast to void*, NULL = default stream) and return; results are valid once the stream
  *     reaches that point.  They never synchronise, never allocate and never wait on device
- *     memory inside a kernel.
+ *     memory inside a kernel.  A sequence of such calls may therefore be captured in a CUDA
+ *     graph (stream capture) and replayed; the replay gives bitwise the eager result.  For
+ *     problems of a few microseconds per step this removes the host's per-call cost.
+ *     (decentlam_step_host_gradients uses a library-owned copy stream and is not meant for
+ *     capture; lsq_grad_static must have been called once outside capture first.)
  *   - All arguments are validated on the host before anything is launched.
  */
 #ifndef DECENTLAM_H_
