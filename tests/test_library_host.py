@@ -250,3 +250,39 @@ def test_gram_argument_validation_on_host():
     assert grad(n=0) == -2 and grad(q=0) == -2 and grad(q=8193) == -8 and grad(n=65536) == -8
     assert grad(x=X + 4) == -3 and grad(H=Hm + 4) == -3
     assert grad(g=X) == -4 and grad(g=Cv) == -4 and grad(g=Hm) == -4
+
+
+def test_header_is_plain_c_and_links_from_c(tmp_path):
+    """include/decentlam.h must be usable from C (not only from the C++ sources that implement it):
+    a C99 program includes it, builds a ring topology on the host, reads its tables back and checks
+    a few weights, linked against the shared library alone."""
+    import os
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "consumer.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include "decentlam.h"
+int main(void) {
+    dlm_topology* t = NULL;
+    const int32_t *rowptr, *col;
+    const float* val;
+    int64_t nnz = 0;
+    int period = 0, n = 0;
+    if (topology_build(DLM_TOPO_RING, 8, NULL, NULL, NULL, &t) != DLM_OK) return 1;
+    if (topology_period(t, &period) != DLM_OK || period != 1) return 2;
+    if (topology_nodes(t, &n) != DLM_OK || n != 8) return 3;
+    if (topology_tables_host(t, 0, &rowptr, &col, &val, &nnz) != DLM_OK || nnz != 24) return 4;
+    if (rowptr[1] != 3 || col[0] != 0 || col[1] != 1 || col[2] != 7) return 5;
+    if (val[1] != (float)(1.0 / 3.0)) return 6;
+    if (decentlam_step(t, 0, 8, 16, 16, NULL, NULL, NULL, DLM_G_F32, 16, 0.9f, 0.1f, NULL) != DLM_ERR_NULL) return 7;
+    printf("%s\n", dlm_status_string(DLM_ERR_TOPOLOGY));
+    return topology_destroy(t) == DLM_OK ? 0 : 8;
+}
+''')
+    exe = tmp_path / "consumer"
+    lib_dir = os.path.dirname(B.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(root, "include"),
+                    str(src), "-o", str(exe), "-L", lib_dir, "-l:libdecentlam.so", f"-Wl,-rpath,{lib_dir}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True)
+    assert out.stdout.strip() == "invalid topology input"
