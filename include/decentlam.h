@@ -147,7 +147,9 @@ DLM_API int topology_destroy(dlm_topology* topo);
  * the "every node i" loops of Algorithms 1 and 2 prescribe), although x and m are
  * overwritten.  All arithmetic is fp32.  Traffic: x, m, g read once, x, m written once.
  * Fastest path: x, m, g 16-byte aligned, ld and ldg multiples of 4 (8 for bf16 g).  Other
- * layouts take a slower scalar path; pointers need only element alignment.
+ * layouts take a scalar path at about half the bandwidth (pad the row stride instead);
+ * pointers need only element alignment.  d may exceed 2^31 (the step is then cut into column
+ * ranges internally, which is exact because the rules are column-wise).
  * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS, DLM_ERR_HYPER,
  *         DLM_ERR_KIND, DLM_ERR_UNSUPPORTED, DLM_ERR_CUDA.
  * ------------------------------------------------------------------------------------ */

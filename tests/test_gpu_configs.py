@@ -158,3 +158,45 @@ def test_node_average_invariant_on_full_tensors(cfg):
             ex = (x.double().mean(0) - xbar_want).abs().max().item() / x.abs().max().item()
             assert em <= 2e-7 and ex <= 2e-7, (cfg, rule, k, em, ex)
             del g
+
+
+@pytest.mark.parametrize("pad", [1, 0])
+@pytest.mark.parametrize("rule", ["decentlam", "dmsgd", "pmsgd"])
+def test_more_than_2_31_columns(rule, pad):
+    """Maximum sizes: d = 2^31 + 4099 columns (n = 2, complete graph, 17 GB per array).  Column
+    indices no longer fit 32 bits and every access to row 1 lies beyond 2^31 elements.
+    pad = 1: row stride d + 1 (a multiple of 4, rows 16-byte aligned): the step is cut into column
+    ranges of 2^30 so that the bulk-copy pipeline's 32-bit tile coordinates stay valid, and the last
+    d mod 4 columns go to the scalar kernel.  pad = 0: odd row stride, rows not 16-byte aligned: the
+    scalar plain-load kernel does everything with 64-bit column indices.
+    One step, checked on sampled columns: both ends, the ragged tail and the neighbourhoods of the
+    range boundaries."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    n, d = 2, (1 << 31) + 4099
+    topo, Ws = build_both("complete", n)
+
+    def draw(std, seed):
+        full = torch.empty((n, d + pad), device=dev)
+        inputs.normal_torch((n, d + pad), std, seed, dev, out=full)
+        return full[:, :d]
+
+    x, m, g = draw(0.02, 91), draw(0.01, 92), draw(1e-3, 93)
+    assert x.stride(0) == d + pad
+    rng = np.random.Generator(np.random.Philox(94))
+    cols = np.unique(np.concatenate([np.arange(0, 4096), np.arange(d - 8200, d), np.arange((1 << 31) - 2048, (1 << 31) + 2048),
+                                     np.arange((1 << 30) - 2048, (1 << 30) + 2048), rng.integers(0, d, 20000)]))
+    idx = torch.from_numpy(cols).to(dev)
+    x0, m0, g0 = to64(x[:, idx]), to64(m[:, idx]), to64(g[:, idx])
+    beta, gamma = np.float32(0.9), np.float32(0.1)
+    if rule == "pmsgd":
+        B.pmsgd_step(x, m, g, float(beta), float(gamma))
+    else:
+        lib_rule(rule, topo, 0, x, m, g, float(beta), float(gamma))
+    torch.cuda.synchronize()
+    assert B.kernel_error() == 0
+    xo, mo = oracle_rule(rule, Ws[0], x0, m0, g0, beta, gamma)
+    assert rel_l2(to64(x[:, idx]), xo) <= 1e-6
+    assert rel_l2(to64(m[:, idx]), mo) <= 1e-6
+    # no sampled column was skipped: untouched columns would still hold their initial values
+    assert not np.array_equal(to64(x[:, idx]), x0)
