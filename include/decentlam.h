@@ -323,7 +323,7 @@ DLM_API int dlm_kernel_error(int* flag);
  *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
  *           size, else none)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
- * the default on rows of 12 or more entries) arranges the same sum differently and
+ * the default on long rows: 12 or more entries, 8 or more for dmsgd_step and up to 128 nodes) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);

@@ -517,14 +517,28 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
     const int lane = threadIdx.x & 31, gbase = lane & ~(L - 1), glane = lane & (L - 1);
     const uint32_t row_bytes = (uint32_t)C * 4;
 
+    constexpr int kPre = 4;  // pass-1 items per thread whose m is fetched ahead (all of them at 512 threads)
     for (long long it = 0; it < my_tiles; ++it) {
+        const long long tile_base = (first + it * gridDim.x) * C;
+        // DmSGD reads m in pass 1, straight from global memory: issue those loads before waiting for
+        // the tile, so that their latency hides behind the copies instead of stalling every item
+        Pack<4> mpre[kPre];
+        if (RULE == DLM_RULE_DMSGD) {
+#pragma unroll
+            for (int k = 0; k < kPre; ++k) {
+                const int e = threadIdx.x + k * blockDim.x;
+                const long long c = tile_base + (e & cv_mask) * 4;
+                mpre[k] = {{0.f, 0.f, 0.f, 0.f}};
+                if (e < items && c < a.d) mpre[k] = ld_f32<4>(a.m + (size_t)(e >> geo.cv_shift) * a.ld + c);
+            }
+        }
         if (!cta_wait(bar, (uint32_t)(it & 1))) {  // uniform decision: give up together
             if (threadIdx.x == 0) atomicExch(&g_kernel_error, 3);
             return;                          // single stage: no other copy of this CTA is in flight
         }
-        const long long tile_base = (first + it * gridDim.x) * C;
         if (RULE != DLM_RULE_DSGD_AWC) {  // pass 1 (the adapt-with-combine rule averages x as it is)
-            for (int e = threadIdx.x; e < items; e += blockDim.x) {
+            int k = 0;
+            for (int e = threadIdx.x; e < items; e += blockDim.x, ++k) {
                 const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
                 const Pack<4> xi = ld_f32<4>(xs + i * C + off);
                 const Pack<4> gi = ld_g<4>(gs + i * C + off);
@@ -536,7 +550,11 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
                 } else if (RULE == DLM_RULE_DMSGD) {  // m' = beta m + g ; y = x - gamma m'
                     const long long c = tile_base + off;
                     Pack<4> mi = {{0.f, 0.f, 0.f, 0.f}}, mn;
-                    if (c < a.d) mi = ld_f32<4>(a.m + (size_t)i * a.ld + c);
+                    if (k < kPre) {
+                        mi = k == 0 ? mpre[0] : k == 1 ? mpre[1] : k == 2 ? mpre[2] : mpre[3];
+                    } else if (c < a.d) {
+                        mi = ld_f32<4>(a.m + (size_t)i * a.ld + c);
+                    }
 #pragma unroll
                     for (int u = 0; u < 4; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], v.v[u]);
                     if (c < a.d) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
@@ -873,12 +891,17 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// Rows of 12 or more entries take the merged-staging kernel when the shape allows it (measured on
-// B200 at n = 256: 9-entry rows are faster with the plain loop, ~14-entry rows with merged staging);
-// everything else the pipeline kernel with the plain mixing loop.
+// Long rows take the merged-staging kernel when the shape allows it, everything else the pipeline
+// kernel with the plain mixing loop.
 template <int RULE, typename GT>
 int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
-    const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : a.max_degree >= 12;
+    // Which mixing pass: measured on ring / exponential / Erdos-Renyi / complete graphs of 32 .. 256 nodes.
+    // Merged staging wins on long or uneven rows; the plain loop on short uniform ones.  DmSGD stages a
+    // single array either way and gains from the merged pass already at 8 entries per row.
+    bool want_merged = a.max_degree >= 12 || (a.max_degree >= 8 && a.n <= 128);
+    if (a.n > 128 && (long long)a.nnz < 8LL * a.n) want_merged = false;
+    if (RULE == DLM_RULE_DMSGD) want_merged = a.max_degree >= 8;
+    const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : want_merged;
     if (merged) {
         int rc = launch_merged<RULE, GT>(a, stream);
         if (rc != DLM_ERR_UNSUPPORTED) return rc;
