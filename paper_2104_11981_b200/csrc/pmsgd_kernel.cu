@@ -59,62 +59,115 @@ __device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
     return {{__uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short*>(p)) << 16)}};
 }
 
+// One pass over the columns [c, c + VEC) of all rows.
+template <typename GT, int VEC>
+__device__ __forceinline__ void pmsgd_columns(int n, long long c, long long ld, float* x, float* m, const GT* g,
+                                              long long ldg, float beta, float gamma) {
+    float sum[VEC];
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) sum[u] = 0.0f;
+    int i = 0;
+    for (; i + kUnroll <= n; i += kUnroll) {  // batches of independent loads, summed in row order
+        Pack<VEC> t[kUnroll];
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r) t[r] = ld_g<VEC>(g + (size_t)(i + r) * ldg + c);
+#pragma unroll
+        for (int r = 0; r < kUnroll; ++r)
+#pragma unroll
+            for (int u = 0; u < VEC; ++u) sum[u] += t[r].v[u];
+    }
+    for (; i < n; ++i) {
+        Pack<VEC> t = ld_g<VEC>(g + (size_t)i * ldg + c);
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) sum[u] += t.v[u];
+    }
+    float gbar[VEC];
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) gbar[u] = sum[u] / (float)n;
+    i = 0;
+    for (; i + kUnroll / 2 <= n; i += kUnroll / 2) {
+        Pack<VEC> xi[kUnroll / 2], mi[kUnroll / 2];
+#pragma unroll
+        for (int r = 0; r < kUnroll / 2; ++r) {
+            xi[r] = ld_f32<VEC>(x + (size_t)(i + r) * ld + c);
+            mi[r] = ld_f32<VEC>(m + (size_t)(i + r) * ld + c);
+        }
+#pragma unroll
+        for (int r = 0; r < kUnroll / 2; ++r) {
+#pragma unroll
+            for (int u = 0; u < VEC; ++u) {
+                mi[r].v[u] = fmaf(beta, mi[r].v[u], gbar[u]);
+                xi[r].v[u] = fmaf(-gamma, mi[r].v[u], xi[r].v[u]);
+            }
+            st_f32<VEC>(m + (size_t)(i + r) * ld + c, mi[r]);
+            st_f32<VEC>(x + (size_t)(i + r) * ld + c, xi[r]);
+        }
+    }
+    for (; i < n; ++i) {
+        Pack<VEC> xi = ld_f32<VEC>(x + (size_t)i * ld + c), mi = ld_f32<VEC>(m + (size_t)i * ld + c);
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) {
+            mi.v[u] = fmaf(beta, mi.v[u], gbar[u]);
+            xi.v[u] = fmaf(-gamma, mi.v[u], xi.v[u]);
+        }
+        st_f32<VEC>(m + (size_t)i * ld + c, mi);
+        st_f32<VEC>(x + (size_t)i * ld + c, xi);
+    }
+}
+
 template <typename GT, int VEC>
 __global__ void __launch_bounds__(kThreads) pmsgd_kernel(int n, long long d, long long ld, float* x, float* m,
                                                           const GT* g, long long ldg, float beta, float gamma) {
     const long long groups = d / VEC;
     for (long long grp = (long long)blockIdx.x * kThreads + threadIdx.x; grp < groups;
-         grp += (long long)gridDim.x * kThreads) {
-        const long long c = grp * VEC;
-        float sum[VEC];
+         grp += (long long)gridDim.x * kThreads)
+        pmsgd_columns<GT, VEC>(n, grp * VEC, ld, x, m, g, ldg, beta, gamma);
+}
+
+// One or two nodes: a thread's single column group has too few bytes in flight (three or six 16-byte
+// loads), so it takes four groups, a block apart (coalesced), with all their gradient loads issued
+// before the first use.  Arithmetic per element is that of pmsgd_columns.
+template <typename GT, int N>
+__global__ void __launch_bounds__(kThreads) pmsgd_few_nodes_kernel(long long d, long long ld, float* x, float* m,
+                                                                    const GT* g, long long ldg, float beta,
+                                                                    float gamma) {
+    constexpr int G = 4;
+    constexpr int n = N;
+    const long long groups = d / 4;
+    const long long first = (long long)blockIdx.x * (G * kThreads) + threadIdx.x;
+    Pack<4> gv[G][N], xv[G][N], mv[G][N];
 #pragma unroll
-        for (int u = 0; u < VEC; ++u) sum[u] = 0.0f;
-        int i = 0;
-        for (; i + kUnroll <= n; i += kUnroll) {  // batches of independent loads, summed in row order
-            Pack<VEC> t[kUnroll];
+    for (int k = 0; k < G; ++k) {
+        const long long grp = first + (long long)k * kThreads;
+        if (grp < groups)
 #pragma unroll
-            for (int r = 0; r < kUnroll; ++r) t[r] = ld_g<VEC>(g + (size_t)(i + r) * ldg + c);
-#pragma unroll
-            for (int r = 0; r < kUnroll; ++r)
-#pragma unroll
-                for (int u = 0; u < VEC; ++u) sum[u] += t[r].v[u];
-        }
-        for (; i < n; ++i) {
-            Pack<VEC> t = ld_g<VEC>(g + (size_t)i * ldg + c);
-#pragma unroll
-            for (int u = 0; u < VEC; ++u) sum[u] += t.v[u];
-        }
-        float gbar[VEC];
-#pragma unroll
-        for (int u = 0; u < VEC; ++u) gbar[u] = sum[u] / (float)n;
-        i = 0;
-        for (; i + kUnroll / 2 <= n; i += kUnroll / 2) {
-            Pack<VEC> xi[kUnroll / 2], mi[kUnroll / 2];
-#pragma unroll
-            for (int r = 0; r < kUnroll / 2; ++r) {
-                xi[r] = ld_f32<VEC>(x + (size_t)(i + r) * ld + c);
-                mi[r] = ld_f32<VEC>(m + (size_t)(i + r) * ld + c);
+            for (int i = 0; i < n; ++i) {
+                gv[k][i] = ld_g<4>(g + (size_t)i * ldg + grp * 4);
+                xv[k][i] = ld_f32<4>(x + (size_t)i * ld + grp * 4);
+                mv[k][i] = ld_f32<4>(m + (size_t)i * ld + grp * 4);
             }
+    }
 #pragma unroll
-            for (int r = 0; r < kUnroll / 2; ++r) {
+    for (int k = 0; k < G; ++k) {
+        const long long grp = first + (long long)k * kThreads;
+        if (grp >= groups) continue;
+        float gbar[4];
 #pragma unroll
-                for (int u = 0; u < VEC; ++u) {
-                    mi[r].v[u] = fmaf(beta, mi[r].v[u], gbar[u]);
-                    xi[r].v[u] = fmaf(-gamma, mi[r].v[u], xi[r].v[u]);
-                }
-                st_f32<VEC>(m + (size_t)(i + r) * ld + c, mi[r]);
-                st_f32<VEC>(x + (size_t)(i + r) * ld + c, xi[r]);
-            }
+        for (int u = 0; u < 4; ++u) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < n; ++i) sum += gv[k][i].v[u];
+            gbar[u] = sum / (float)n;
         }
-        for (; i < n; ++i) {
-            Pack<VEC> xi = ld_f32<VEC>(x + (size_t)i * ld + c), mi = ld_f32<VEC>(m + (size_t)i * ld + c);
 #pragma unroll
-            for (int u = 0; u < VEC; ++u) {
-                mi.v[u] = fmaf(beta, mi.v[u], gbar[u]);
-                xi.v[u] = fmaf(-gamma, mi.v[u], xi.v[u]);
+        for (int i = 0; i < n; ++i) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                mv[k][i].v[u] = fmaf(beta, mv[k][i].v[u], gbar[u]);
+                xv[k][i].v[u] = fmaf(-gamma, mv[k][i].v[u], xv[k][i].v[u]);
             }
-            st_f32<VEC>(m + (size_t)i * ld + c, mi);
-            st_f32<VEC>(x + (size_t)i * ld + c, xi);
+            st_f32<4>(m + (size_t)i * ld + grp * 4, mv[k][i]);
+            st_f32<4>(x + (size_t)i * ld + grp * 4, xv[k][i]);
         }
     }
 }
@@ -130,6 +183,15 @@ int launch(int n, int64_t d, int64_t ld, float* x, float* m, const GT* g, int64_
     long long groups = d / VEC;
     long long blocks = (groups + kThreads - 1) / kThreads;
     long long cap = g_pmsgd_tune_cap > 0 ? (long long)sms * g_pmsgd_tune_cap : 0x7fffffffLL;
+    if (VEC == 4 && n <= 2 && g_pmsgd_tune_cap <= 0) {
+        blocks = (groups + 4 * kThreads - 1) / (4 * kThreads);
+        if (n == 1)
+            pmsgd_few_nodes_kernel<GT, 1><<<(unsigned)blocks, kThreads, 0, s>>>(d, ld, x, m, g, ldg, beta, gamma);
+        else
+            pmsgd_few_nodes_kernel<GT, 2><<<(unsigned)blocks, kThreads, 0, s>>>(d, ld, x, m, g, ldg, beta, gamma);
+        dlm_count_launch(1);
+        return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+    }
     if (blocks > cap) blocks = cap;
     pmsgd_kernel<GT, VEC><<<(unsigned)blocks, kThreads, 0, s>>>(n, d, ld, x, m, g, ldg, beta, gamma);
     dlm_count_launch(1);

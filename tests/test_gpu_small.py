@@ -237,3 +237,11 @@ def test_extreme_node_counts(rule, n, topology, d):
     fits in shared memory (complete graphs: 256 or 512 entries per row), and the degenerate n = 1
     (W = [1]: plain momentum SGD) and n = 2."""
     _case(rule, topology, n, d, "f32", seed=n + d, steps=2)
+
+
+@pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,d", [(1, 5000), (2, 100_003), (2, 4 * 1024 * 5 + 8), (1, 4096)])
+def test_pmsgd_with_one_or_two_nodes(n, d, g_dtype):
+    """PmSGD on one or two nodes takes a kernel of its own (four column groups per thread): whole
+    blocks, a ragged last block and the scalar tail, with padded rows and canaries."""
+    _case("pmsgd", "complete", n, d, g_dtype, ld=d + (8 - d % 8) % 8 + 8, offset=8, seed=3 * n + d % 97, steps=2)
