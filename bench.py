@@ -45,16 +45,16 @@ def parse_args():
     return ap.parse_args()
 
 
-# DRAM counters of step_tma_kernel<DecentLaM, fp32 g> from the ncu capture summarised in
-# profiles/step_tma_kernel_decentlam_n16_d2M.md (n = 16, 2,097,152 columns), per node-parameter.
+# DRAM counters of step_tma_kernel<DecentLaM, fp32 g> from the ncu launch list summarised in
+# profiles/kernels_n16_d2M_traffic.md (n = 16, 2,097,152 columns), per node-parameter.
 # Valid only for the kernel source they were taken from: reported while the source file's
 # SHA-256 matches, otherwise "traffic" is null.
 NCU_CAPTURE = {
     "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
-    "sha256": "4bd2ade38e6ff427d2124ab76716e08d46c6050e95943d9a129cbd53e4d9913c",
+    "sha256": "db033466c94e16bbdb1255116add8bb028bd8bd117172e3164068a620397a153",
     "workload": "cfg2",
     "dram_read_bytes_per_np": 402.70e6 / (16 * 2097152),
-    "dram_write_bytes_per_np": 211.62e6 / (16 * 2097152),
+    "dram_write_bytes_per_np": 211.59e6 / (16 * 2097152),
 }
 
 

@@ -463,6 +463,7 @@ struct MergedGeom {
     int C;          // tile columns (power of two, 32 .. 256)
     int cv_shift;   // log2(C / 4)
     int tables_in_smem;
+    int prefetch_m;        // DecentLaM: request the tile's m lines into L2 before waiting for the tile
     uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
     uint32_t v_off, g_off; // byte offsets of the staged-value tile and of the g landing area inside the stage
     uint32_t stage_bytes;
@@ -532,6 +533,18 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
                 if (e < items && c < a.d) mpre[k] = ld_f32<4>(a.m + (size_t)(e >> geo.cv_shift) * a.ld + c);
             }
         }
+        if (LAM && geo.prefetch_m) {
+            // DecentLaM reads m in pass 2, one load per item just before its mixing loop, too short a loop
+            // to cover a trip to DRAM.  Ask for those lines now, while the tile is still on its way: the
+            // prefetch holds no registers and the later load finds its line in L2.  One request for each
+            // end of every 128-byte row segment (a segment may straddle two lines).
+            const int seg_shift = geo.cv_shift - 3, segs = a.n << seg_shift;  // C / 32 segments per row
+            for (int e = threadIdx.x; e < 2 * segs; e += blockDim.x) {
+                const int sg = e >> 1;
+                const long long c = tile_base + (long long)(sg & ((1 << seg_shift) - 1)) * 32 + (e & 1) * 28;
+                if (c < a.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.m + (size_t)(sg >> seg_shift) * a.ld + c));
+            }
+        }
         if (!cta_wait(bar, (uint32_t)(it & 1))) {  // uniform decision: give up together
             if (threadIdx.x == 0) atomicExch(&g_kernel_error, 3);
             return;                          // single stage: no other copy of this CTA is in flight
@@ -595,7 +608,9 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
                     en = ent[ri.y + base0 + glane];
                     if (!LAM && en.x == i) en.y = self_bits;
                 }
-                const int cnt = min(L, (len_max - base0 + 3) & ~3);
+                // DecentLaM keeps whole groups of four (no remainder loop: its m loads are in flight and
+                // registers are short); the averaging rules stop at the longest row of the warp
+                const int cnt = LAM ? min(L, (len_max - base0 + 3) & ~3) : min(L, len_max - base0);
 #pragma unroll 4
                 for (int r = 0; r < cnt; ++r) {
                     const int j = __shfl_sync(full, en.x, gbase + r);
@@ -876,6 +891,9 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     }
     geo.C = C;
     geo.cv_shift = ilog2(C / 4);
+    // measured: +3 to +8 % with tiles of 64 columns or more (up to 128 nodes); with 256 nodes and
+    // 32-column tiles the extra requests cost 6 % instead
+    geo.prefetch_m = C >= 64;
     geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
     geo.num_tiles = (a.d + C - 1) / C;
     CUtensorMap tm_x, tm_g;
@@ -902,6 +920,9 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     bool want_merged = a.max_degree >= 12 || (a.max_degree >= 8 && a.n <= 128);
     if (a.n > 128 && (long long)a.nnz < 8LL * a.n) want_merged = false;
     if (RULE == DLM_RULE_DMSGD) want_merged = a.max_degree >= 8;
+    // one staged array and no momentum in pass 2: up to 128 nodes DmSGD and adapt-then-combine DSGD gain
+    // 1 to 7 % from six entries per row on (exponential graphs of 32 and 64 nodes)
+    if ((RULE == DLM_RULE_DMSGD || RULE == DLM_RULE_DSGD_ATC) && a.n <= 128 && a.max_degree >= 6) want_merged = true;
     const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : want_merged;
     if (merged) {
         int rc = launch_merged<RULE, GT>(a, stream);
