@@ -48,6 +48,7 @@ __device__ __forceinline__ void dmsgd_local(float xi, float mi, float gi, float 
     y = fmaf(-gamma, mn, xi);
 }
 
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
 
 template <int VEC>
@@ -96,14 +97,30 @@ __device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
 
 
 // Neighbour tables of the current slot, either copied to shared memory or left in global memory.
-struct Tables {
+// DecentLaM reads packed entries {column, bits of the weight}, one 64-bit load per neighbour (3.6 % on
+// the 64-node bf16 workload); the averaging rules read separate column and weight arrays, which keeps
+// the DSGD kernels at 40 registers, i.e. six CTAs per SM (with packed entries: 49 registers, 13 % slower).
+template <bool PACKED>
+struct Tables;
+template <>
+struct Tables<false> {
     const int* rowptr;
     const int* col;
     const float* val;
     const int* order;
 };
+template <>
+struct Tables<true> {
+    const int* rowptr;
+    const int2* ent;
+    const int* order;
+};
 
-__device__ __forceinline__ Tables stage_tables(const dlm_step_args& a, void* smem_tables, bool in_smem) {
+// smem_tables must be 8-byte aligned.
+template <bool PACKED>
+__device__ __forceinline__ Tables<PACKED> stage_tables(const dlm_step_args& a, void* smem_tables, bool in_smem);
+template <>
+__device__ __forceinline__ Tables<false> stage_tables<false>(const dlm_step_args& a, void* smem_tables, bool in_smem) {
     if (!in_smem) return {a.rowptr, a.col, a.val, a.order};
     int* s_rowptr = reinterpret_cast<int*>(smem_tables);
     int* s_order = s_rowptr + (a.n + 1);
@@ -117,11 +134,23 @@ __device__ __forceinline__ Tables stage_tables(const dlm_step_args& a, void* sme
     }
     return {s_rowptr, s_col, s_val, s_order};
 }
+template <>
+__device__ __forceinline__ Tables<true> stage_tables<true>(const dlm_step_args& a, void* smem_tables, bool in_smem) {
+    const int2* ent = reinterpret_cast<const int2*>(a.ent);
+    if (!in_smem) return {a.rowptr, ent, a.order};
+    int2* s_ent = reinterpret_cast<int2*>(smem_tables);
+    int* s_rowptr = reinterpret_cast<int*>(s_ent + a.nnz);
+    int* s_order = s_rowptr + (a.n + 1);
+    for (int i = threadIdx.x; i <= a.n; i += blockDim.x) s_rowptr[i] = a.rowptr[i];
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s_order[i] = a.order[i];
+    for (int i = threadIdx.x; i < a.nnz; i += blockDim.x) s_ent[i] = ent[i];
+    return {s_rowptr, s_ent, s_order};
+}
 
 // Mix one item (row i, VEC consecutive columns at tile offset off) of the DecentLaM rule.
 //   xs, gs: staged tiles [n][C] (gs may hold bf16 when GS is __nv_bfloat16)
 template <int VEC, typename GS>
-__device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, int C, const float* xs,
+__device__ __forceinline__ void decentlam_item(const Tables<true>& t, int i, int off, int C, const float* xs,
                                                const GS* gs, const Pack<VEC>& mi, float beta, float gamma,
                                                float inv_gamma, Pack<VEC>& mn, Pack<VEC>& xn) {
     const Pack<VEC> xi = ld_f32<VEC>(xs + i * C + off);
@@ -130,8 +159,9 @@ __device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, 
     for (int u = 0; u < VEC; ++u) mixg[u] = cons[u] = 0.0f;
     const int p1 = t.rowptr[i + 1];
     for (int p = t.rowptr[i]; p < p1; ++p) {  // neighbours in ascending order
-        const int j = t.col[p];
-        const float w = t.val[p];
+        const int2 en = t.ent[p];
+        const int j = en.x;
+        const float w = __int_as_float(en.y);
         const Pack<VEC> gj = ld_g<VEC>(gs + j * C + off);
 #pragma unroll
         for (int u = 0; u < VEC; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
@@ -148,7 +178,7 @@ __device__ __forceinline__ void decentlam_item(const Tables& t, int i, int off, 
 
 // Partial average of the DmSGD rule on staged y = x - gamma m':  x' = y_i + sum_{j != i} w_ij (y_j - y_i)
 template <int VEC>
-__device__ __forceinline__ void dmsgd_item(const Tables& t, int i, int off, int C, const float* ys,
+__device__ __forceinline__ void dmsgd_item(const Tables<false>& t, int i, int off, int C, const float* ys,
                                            Pack<VEC>& xn) {
     const Pack<VEC> yi = ld_f32<VEC>(ys + i * C + off);
     float acc[VEC];
@@ -177,13 +207,14 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* gs = xs + (size_t)a.n * C;
-    void* tab = (RULE == DLM_RULE_DECENTLAM) ? (void*)(gs + (size_t)a.n * C) : (void*)gs;
+    unsigned char* tab = reinterpret_cast<unsigned char*>((RULE == DLM_RULE_DECENTLAM) ? gs + (size_t)a.n * C : gs);
+    tab += (8u - (smem_u32(tab) & 7u)) & 7u;  // 64-bit table entries (a scalar tile may end on a 4-byte boundary)
     // This kernel serves the small, latency-bound problems and is launched with programmatic
     // stream serialization: it may be scheduled while its predecessor drains and waits here until
     // that grid has completed and its writes are visible (the tables never change, so staging
     // them would be safe earlier, but they are tiny).
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const Tables t = stage_tables(a, tab, tables_in_smem != 0);
+    const auto t = stage_tables<RULE == DLM_RULE_DECENTLAM>(a, tab, tables_in_smem != 0);
     const GT* g = reinterpret_cast<const GT*>(a.g);
     const int items = a.n << cv_shift;
     const int cv_mask = (1 << cv_shift) - 1;
@@ -223,7 +254,7 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
             const long long c = c_base + off;
             if (c < a.d) {
                 Pack<VEC> xn;
-                if (RULE == DLM_RULE_DECENTLAM) {
+                if constexpr (RULE == DLM_RULE_DECENTLAM) {
                     const Pack<VEC> mi = ld_f32<VEC>(a.m + (size_t)i * a.ld + c);
                     Pack<VEC> mn;
                     decentlam_item<VEC, float>(t, i, off, C, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
@@ -247,7 +278,6 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
 // Shared memory per stage: x tile [n][C] fp32 | m tile [n][C] fp32 | g tile [n][C] GT, each
 // rounded up to 128 bytes; then `stages` mbarriers; then the tables.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -343,7 +373,7 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         for (int s = 0; s < geo.stages && s < my_tiles; ++s) issue(s, first + (long long)s * gridDim.x);
     }
     // tables staged in shared memory when small, else read from global memory (cached)
-    const Tables t = stage_tables(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
+    const auto t = stage_tables<RULE == DLM_RULE_DECENTLAM>(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
     __syncthreads();  // barriers initialised and tables staged for everyone
 
     for (long long it = 0; it < my_tiles; ++it) {
@@ -403,7 +433,7 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
                 const long long c = c_base + off;
                 if (c < a.d) {  // columns past d hold the copies' zero fill
                     Pack<4> xn;
-                    if (RULE == DLM_RULE_DECENTLAM) {
+                    if constexpr (RULE == DLM_RULE_DECENTLAM) {
                         const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
                         Pack<4> mn;
                         decentlam_item<4, GT>(t, i, off, Cb, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
