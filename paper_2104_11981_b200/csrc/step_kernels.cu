@@ -6,12 +6,16 @@
 // and only then writes x and m of the same tile.  This makes the in-place update exact
 // (simultaneous update of all nodes) with each of x, m, g read once and x, m written once.
 //
-// Two implementations of the same arithmetic:
-//   step_tma_kernel   persistent CTAs, multi-stage pipeline of 2-D tensor bulk copies
-//                     (cp.async.bulk.tensor) completing on mbarriers; needs 16-byte aligned rows.
-//   step_tile_kernel  plain vector/scalar loads into shared memory; any alignment, any n,
-//                     also used for the last d mod 4 columns.
-// Both call the same per-element update functions, so their results are bitwise identical.
+// Three kernels:
+//   step_tma_kernel     the tile arrives by 2-D tensor bulk copies (cp.async.bulk.tensor) completing on an
+//                       mbarrier; by default one stage per CTA and a grid of many short-lived CTAs, several
+//                       resident per SM (a persistent multi-stage pipeline is selectable).  Needs 16-byte
+//                       aligned rows and n <= 256.
+//   step_tile_kernel    plain vector/scalar loads into shared memory; any alignment, n up to 2048, also
+//                       used for tiny problems and for the last d mod 4 columns.
+//   step_merged_kernel  for long neighbour lists: one staged value per neighbour (see its own header).
+// The first two call the same per-element update functions, so their results are bitwise identical; the
+// third evaluates the same sums in another arrangement and agrees with them to rounding.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
