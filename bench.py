@@ -51,10 +51,10 @@ def parse_args():
 # SHA-256 matches, otherwise "traffic" is null.
 NCU_CAPTURE = {
     "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
-    "sha256": "4096166dd6c6a2138760248ea19878387f509baab0b787f2d3fd4e6039aab0a7",
+    "sha256": "66b9f05b4ce2bd9402c7d14764ad35995ed4cdd64a822f9ce08b51e80c6cc696",
     "workload": "cfg2",
-    "dram_read_bytes_per_np": 402.70e6 / (16 * 2097152),
-    "dram_write_bytes_per_np": 211.57e6 / (16 * 2097152),
+    "dram_read_bytes_per_np": 402.71e6 / (16 * 2097152),
+    "dram_write_bytes_per_np": 211.65e6 / (16 * 2097152),
 }
 
 

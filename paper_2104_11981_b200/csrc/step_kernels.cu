@@ -10,7 +10,7 @@
 //   step_tma_kernel     the tile arrives by 2-D tensor bulk copies (cp.async.bulk.tensor) completing on an
 //                       mbarrier; by default one stage per CTA and a grid of many short-lived CTAs, several
 //                       resident per SM (a persistent multi-stage pipeline is selectable).  Needs 16-byte
-//                       aligned rows and n <= 256.
+//                       aligned rows; more than 256 nodes arrive as several row boxes per array.
 //   step_tile_kernel    plain vector/scalar loads into shared memory; any alignment, n up to 2048, also
 //                       used for tiny problems and for the last d mod 4 columns.
 //   step_merged_kernel  for long neighbour lists: one staged value per neighbour (see its own header).
@@ -330,6 +330,8 @@ struct TmaGeom {
     int C;           // tile columns = boxes * box_cols
     int box_cols;    // columns per bulk copy (power of two, <= 256; 16-byte multiple)
     int boxes;       // bulk copies per array and stage; each lands as a dense [n][box_cols] sub-tile
+    int row_boxes;   // more than 256 nodes: the rows of a tile arrive as row_boxes copies of box_rows rows each
+    int box_rows;    // (a copy's box is at most 256 rows high); only with boxes == 1
     int cv_shift;    // log2(box_cols / 4)
     int stages;
     uint32_t x_bytes, g_bytes, stage_bytes;  // per-stage tile sizes (128-byte multiples)
@@ -363,6 +365,16 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         const uint32_t dst = smem_u32(base + (size_t)s * geo.stage_bytes);
         const int c0 = (int)(tile * C);
         mbar_expect_tx(bar, geo.tx_bytes);
+        if (geo.row_boxes > 1) {  // consecutive row boxes land one after the other: a dense [rows][Cb] tile
+            const uint32_t rb_x = (uint32_t)geo.box_rows * Cb * 4, rb_g = (uint32_t)geo.box_rows * Cb * (uint32_t)sizeof(GT);
+            for (int r = 0; r < geo.row_boxes; ++r) {
+                tma_load_2d(dst + r * rb_x, &tm_x, c0, r * geo.box_rows, bar);
+                tma_load_2d(dst + geo.g_off + r * rb_g, &tm_g, c0, r * geo.box_rows, bar);
+                if (RULE == DLM_RULE_DECENTLAM || RULE == DLM_RULE_DMSGD)
+                    tma_load_2d(dst + geo.m_off + r * rb_x, &tm_m, c0, r * geo.box_rows, bar);
+            }
+            return;
+        }
         for (int b = 0; b < geo.boxes; ++b) {
             tma_load_2d(dst + b * sub_x, &tm_x, c0 + b * Cb, 0, bar);
             tma_load_2d(dst + geo.g_off + b * sub_g, &tm_g, c0 + b * Cb, 0, bar);
@@ -737,14 +749,14 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D map over a row-major [n, d] array with row stride ld elements; box = [n rows, C columns].
-bool make_map(CUtensorMap* map, const void* ptr, bool bf16, int n, int64_t d, int64_t ld, int C) {
+// 2-D map over a row-major [n, d] array with row stride ld elements; box = [n rows (or box_rows), C columns].
+bool make_map(CUtensorMap* map, const void* ptr, bool bf16, int n, int64_t d, int64_t ld, int C, int box_rows = 0) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t esz = bf16 ? 2 : 4;
     cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
     cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
-    cuuint32_t box[2] = {(cuuint32_t)C, (cuuint32_t)n};
+    cuuint32_t box[2] = {(cuuint32_t)C, (cuuint32_t)(box_rows > 0 ? box_rows : n)};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                     const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -815,7 +827,12 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     if (!dev.ok) return DLM_ERR_CUDA;
     const bool bf16 = sizeof(GT) == 2;
     const int min_c = bf16 ? 8 : 4;  // 16-byte inner box extent
-    if (a.n > 256 || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
+    if (a.n > DLM_MAX_NODES || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
+    // A copy's box is at most 256 rows high: more nodes arrive as several row boxes of equal height, a
+    // multiple of 8 rows, so that every box lands on a 128-byte boundary whatever the tile width.
+    const int row_boxes = (a.n + 255) / 256;
+    const int box_rows = row_boxes == 1 ? a.n : (((a.n + row_boxes - 1) / row_boxes + 7) & ~7);
+    const size_t n_pad = (size_t)row_boxes * box_rows;  // rows past n are filled with zeros and never read
     const size_t tab = table_bytes(a);
     // Small tables are staged in shared memory by every CTA; large ones stay in global memory
     // (all CTAs read the same few KB, so they live in L1/L2).
@@ -824,8 +841,8 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     const size_t budget = (size_t)dev.smem_optin;
     constexpr bool HAS_M = RULE == DLM_RULE_DECENTLAM || RULE == DLM_RULE_DMSGD;
     auto stage_bytes_for = [&](int C, uint32_t& xb, uint32_t& gb) {
-        xb = (uint32_t)(((size_t)a.n * C * 4 + 127) & ~(size_t)127);
-        gb = (uint32_t)(((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127);
+        xb = (uint32_t)((n_pad * C * 4 + 127) & ~(size_t)127);
+        gb = (uint32_t)((n_pad * C * sizeof(GT) + 127) & ~(size_t)127);
         return (size_t)(HAS_M ? 2 : 1) * xb + gb;
     };
     // Defaults (measured on B200): about 16 KB per staged array with row segments of at least
@@ -837,7 +854,17 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     // 6.7 instead of 6.0 TB/s at n = 8, 6.6 instead of 4.4 at n = 4 with single-box tiles).
     int C = 1 << ilog2(std::max(1, (int)(16384 / ((size_t)a.n * 4))));
     C = std::max(std::max(min_c, a.n <= 128 ? 64 : 32), std::min(4096, C));  // 64 columns beat 32 at n = 128
+    if (row_boxes > 1) {
+        // More than 256 nodes (measured at 300 .. 2048 nodes): row segments of 128 bytes if they fit at
+        // all, wider ones only while two CTAs per SM still fit; 512 threads.
+        uint32_t xb0, gb0;
+        int c_fit = 256, c_two = 256;
+        while (c_fit > min_c && stage_bytes_for(c_fit, xb0, gb0) + fixed > budget) c_fit /= 2;
+        while (c_two > min_c && stage_bytes_for(c_two, xb0, gb0) + fixed > budget / 2 - 1024) c_two /= 2;
+        C = std::max(c_two, std::min(32, c_fit));
+    }
     if (g_tune_cols >= min_c && g_tune_cols <= 4096 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
+    if (row_boxes > 1) C = std::min(C, 256);  // row boxes and several column boxes do not combine
     int stages = g_tune_stages > 0 ? std::min(g_tune_stages, kMaxStages) : 1;
     int ctas = g_tune_ctas > 0 ? g_tune_ctas : 1;
     // tiles per CTA: 1 when the per-CTA set-up (table staging) is negligible (up to 2.5 KB of tables:
@@ -855,15 +882,17 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     const int box_cols = std::min(C, 256);
 
     CUtensorMap tm_x, tm_m, tm_g;
-    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, box_cols) ||
-        !make_map(&tm_m, HAS_M ? a.m : a.x, false, a.n, a.d, a.ld, box_cols) ||
-        !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, box_cols))
+    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, box_cols, box_rows) ||
+        !make_map(&tm_m, HAS_M ? a.m : a.x, false, a.n, a.d, a.ld, box_cols, box_rows) ||
+        !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, box_cols, box_rows))
         return DLM_ERR_UNSUPPORTED;
 
     TmaGeom geo;
     geo.C = C;
     geo.box_cols = box_cols;
     geo.boxes = C / box_cols;
+    geo.row_boxes = row_boxes;
+    geo.box_rows = box_rows;
     geo.cv_shift = ilog2(box_cols / 4);
     geo.stages = stages;
     geo.x_bytes = xb;
@@ -871,7 +900,7 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     geo.stage_bytes = (uint32_t)sb;
     geo.m_off = xb;
     geo.g_off = HAS_M ? 2 * xb : xb;
-    geo.tx_bytes = (uint32_t)((size_t)a.n * C * ((HAS_M ? 8 : 4) + sizeof(GT)));
+    geo.tx_bytes = (uint32_t)(n_pad * C * ((HAS_M ? 8 : 4) + sizeof(GT)));
     geo.tables_in_smem = tables_in_smem;
     geo.num_tiles = (a.d + C - 1) / C;
     size_t smem = fixed + (size_t)stages * sb;
@@ -882,7 +911,7 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
                                        : std::min<long long>(geo.num_tiles, (long long)dev.sms * ctas);
     // long neighbour lists need more warps in flight to hide the mixing loop's latency
     const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512)
-                            ? g_tune_threads : (a.max_degree > 8 ? 512 : 256);
+                            ? g_tune_threads : ((a.max_degree > 8 || row_boxes > 1) ? 512 : 256);
     kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_m, tm_g, a, geo);
     dlm_count_launch(1);
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
@@ -962,6 +991,9 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
         int rc = launch_merged<RULE, GT>(a, stream);
         if (rc != DLM_ERR_UNSUPPORTED) return rc;
     }
+    // DmSGD on 257 .. 511 nodes: the plain-load kernel stages one array where the bulk-copy kernel stages
+    // three, and its wider tiles win there (ring of 300 nodes: 4.6 against 4.0 TB/s)
+    if (RULE == DLM_RULE_DMSGD && a.n > 256 && a.n < 512 && g_tune_path != 2) return DLM_ERR_UNSUPPORTED;
     return launch_tma_plain<RULE, GT>(a, stream);
 }
 

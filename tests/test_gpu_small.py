@@ -143,6 +143,37 @@ def test_kernel_paths_agree_bitwise(rule, g_dtype):
             assert not torch.equal(x, outs[0][0])      # it really is the other arithmetic
 
 
+@pytest.mark.parametrize("topology,n,d", [("ring", 257, 4104), ("ring", 300, 8008), ("static_exp", 777, 2056),
+                                          ("ring", 1000, 1032), ("static_exp", 2048, 520)])
+def test_more_than_256_nodes_row_boxes_agree_bitwise(topology, n, d):
+    """Above 256 nodes a tile's rows arrive as several bulk copies (a copy's box is at most 256 rows
+    high; box heights are padded to a multiple of 8 rows, rows past n are zero fill).  Whatever the
+    tile width and block size, the result equals the plain-load kernel's bit for bit."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    topo, _ = build_both(topology, n)
+    for rule in ("decentlam", "dmsgd", "dsgd_atc", "dsgd_awc"):
+        for gt in (torch.float32, torch.bfloat16):
+            x0 = inputs.normal_torch((n, d), 0.02, 1, dev); m0 = inputs.normal_torch((n, d), 0.01, 2, dev)
+            g = inputs.normal_torch((n, d), 1e-3, 3, dev, dtype=gt)
+            outs = []
+            try:
+                # (path, tile columns, threads): plain loads, then bulk copies in the automatic and in forced shapes
+                for path, cols, thr in ((1, 0, 0), (2, 0, 0), (2, 8, 256), (2, 16, 512), (2, 64, 512)):
+                    B.set_tuning(0, path); B.set_tuning(7, 1 if path == 2 else 0); B.set_tuning(1, cols); B.set_tuning(6, thr)
+                    x, m = x0.clone(), m0.clone()
+                    for k in range(2):
+                        lib_rule(rule, topo, k, x, m, g, 0.9, 0.1)
+                    torch.cuda.synchronize()
+                    assert B.kernel_error() == 0
+                    outs.append((x, m))
+            finally:
+                for knob in range(8):
+                    B.set_tuning(knob, 0)
+            for x, m in outs[1:]:
+                assert torch.equal(x, outs[0][0]) and torch.equal(m, outs[0][1]), (rule, gt)
+
+
 @pytest.mark.parametrize("rule", RULES)
 def test_deterministic_and_column_independent(rule):
     """Repeated runs are bitwise identical, and a column range run alone equals that range of the
