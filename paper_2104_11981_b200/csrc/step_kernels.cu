@@ -854,6 +854,13 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     // 6.7 instead of 6.0 TB/s at n = 8, 6.6 instead of 4.4 at n = 4 with single-box tiles).
     int C = 1 << ilog2(std::max(1, (int)(16384 / ((size_t)a.n * 4))));
     C = std::max(std::max(min_c, a.n <= 128 ? 64 : 32), std::min(4096, C));  // 64 columns beat 32 at n = 128
+    // The DSGD rules stage two arrays and need 40 registers: with 128-thread CTAs and tiles of about 8 KB per
+    // array many more CTAs share an SM.  Measured on 4 .. 64 nodes: adapt-with-combine +5 to +17 %;
+    // adapt-then-combine (one more pass and barrier per tile) +17 % on 4 nodes and +19 % with bf16
+    // gradients, but 2 to 4 % slower on 8 .. 32 nodes with fp32 gradients, where it keeps the common shape.
+    constexpr bool DSGD = RULE == DLM_RULE_DSGD_ATC || RULE == DLM_RULE_DSGD_AWC;
+    const bool dsgd_small = DSGD && a.n <= 64 && a.max_degree <= 8 && (RULE == DLM_RULE_DSGD_AWC || bf16 || a.n <= 4);
+    if (dsgd_small) C = std::max(64, 1 << ilog2(std::max(1, (bf16 ? 4096 : 2048) / a.n)));
     if (row_boxes > 1) {
         // More than 256 nodes (measured at 300 .. 2048 nodes): row segments of 128 bytes if they fit at
         // all, wider ones only while two CTAs per SM still fit; 512 threads.
@@ -911,7 +918,7 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
                                        : std::min<long long>(geo.num_tiles, (long long)dev.sms * ctas);
     // long neighbour lists need more warps in flight to hide the mixing loop's latency
     const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512)
-                            ? g_tune_threads : ((a.max_degree > 8 || row_boxes > 1) ? 512 : 256);
+                            ? g_tune_threads : ((a.max_degree > 8 || row_boxes > 1) ? 512 : dsgd_small ? 128 : 256);
     kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_m, tm_g, a, geo);
     dlm_count_launch(1);
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
