@@ -13,7 +13,11 @@ TOL_STEP, TOL_T = 1e-6, 1e-4
 @pytest.mark.parametrize("rule", ["dsgd_atc", "dsgd_awc"])
 @pytest.mark.parametrize("topology,n,d,g_dtype", [("ring", 8, 4096, "f32"), ("one_peer_exp", 16, 300_007, "f32"),
                                                    ("static_exp", 64, 100_000, "bf16"), ("mesh", 16, 65_537, "f32"),
-                                                   ("er_mh", 40, 50_001, "f32"), ("ring", 5, 3, "f32"), ("sym_exp", 8, 1, "bf16")])
+                                                   ("er_mh", 40, 50_001, "f32"), ("ring", 5, 3, "f32"), ("sym_exp", 8, 1, "bf16"),
+                                                   # 16-byte aligned rows, bulk-copy kernel: the 128-thread launch shape of
+                                                   # the DSGD rules (adapt-with-combine; 4 nodes; bf16 gradients) and the common one
+                                                   ("one_peer_exp", 16, 300_008, "f32"), ("ring", 4, 1_000_008, "f32"),
+                                                   ("one_peer_exp", 16, 300_008, "bf16"), ("mesh", 64, 50_008, "f32")])
 def test_dsgd_matches_oracle(rule, topology, n, d, g_dtype):
     dev = torch.device("cuda:0")
     topo, Ws = build_both(topology, n, graph_seed=5, er_p=0.3)
