@@ -39,37 +39,54 @@ def parse_args():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--columns", type=int, default=0,
                     help="override d (columns per node): a smaller case of the same kernel, for profiler captures")
+    ap.add_argument("--sharded", type=int, default=0,
+                    help="node-sharded run over this many ranks (the paper's deployment): under torchrun with --gpus N "
+                         "ranks exchange halo rows over NCCL; on one GPU rank 0's share is timed with device copies "
+                         "standing in for the link")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the DmSGD / PmSGD side timings")
     return ap.parse_args()
 
 
-# DRAM counters of step_tma_kernel<DecentLaM, fp32 g> from the ncu launch list summarised in
-# profiles/kernels_n16_d2M_traffic.md (n = 16, 2,097,152 columns), per node-parameter.
-# Valid only for the kernel source they were taken from: reported while the source file's
-# SHA-256 matches, otherwise "traffic" is null.
+# DRAM counters of step_tma_kernel<DecentLaM, fp32 g> from an ncu capture of this very program on a smaller
+# case of the benchmarked kernel (16 nodes, `--columns 8388608`; three metrics only: duration, DRAM bytes
+# read, DRAM bytes written).  Reads scale with the columns.  Writes do too, except for the lines still
+# sitting in the L2 when the kernel ends: that residue does not grow with the problem (the same number of
+# bytes at 2,097,152 and at 8,388,608 columns), so it is carried over as a constant, not scaled.
+# Valid only for the kernel sources they were taken from: reported while their SHA-256 matches, else null.
 NCU_CAPTURE = {
-    "source": os.path.join("paper_2104_11981_b200", "csrc", "step_kernels.cu"),
-    "sha256": "36cf71200973c161f9075fd02147594a102c2fe998b725a116e0145a28dbec25",
+    "sources": [os.path.join("paper_2104_11981_b200", "csrc", f) for f in ("step_kernels.cu", "dlm_device.cuh")],
+    "sha256": "4193107fb7e907e44b02b0c4fb78fc28b170eda131eeff60d644643e49de19ce",
     "workload": "cfg2",
-    "dram_read_bytes_per_np": 402.71e6 / (16 * 2097152),
-    "dram_write_bytes_per_np": 211.61e6 / (16 * 2097152),
+    "capture_units": 16 * 8388608,
+    "dram_read_bytes": 1610689152.0,     # mean of two captured launches (1,610,672,640 and 1,610,705,664)
+    "dram_write_bytes": 1015718528.0,    # mean of two captured launches (1,017,510,912 and 1,013,926,144)
 }
 
 
 def ncu_traffic(workload, units):
-    """DRAM bytes per launch scaled from the small-case capture by the units processed, or None."""
+    """DRAM bytes per launch of the benchmarked size, from the small-case capture: (dict, total) or (None, None)."""
     import hashlib
-    if workload != NCU_CAPTURE["workload"]:
-        return None
+    if workload != NCU_CAPTURE["workload"] or not NCU_CAPTURE["sha256"]:
+        return None, None
     try:
-        with open(os.path.join(ROOT, NCU_CAPTURE["source"]), "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest() != NCU_CAPTURE["sha256"]:
-                return None
+        h = hashlib.sha256()
+        for src in NCU_CAPTURE["sources"]:
+            with open(os.path.join(ROOT, src), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest() != NCU_CAPTURE["sha256"]:
+            return None, None
     except OSError:
-        return None
-    return (NCU_CAPTURE["dram_read_bytes_per_np"] + NCU_CAPTURE["dram_write_bytes_per_np"]) * units
+        return None, None
+    cu = NCU_CAPTURE["capture_units"]
+    reads = NCU_CAPTURE["dram_read_bytes"] / cu * units
+    residue = 8.0 * cu - NCU_CAPTURE["dram_write_bytes"]          # written lines still in L2 when the capture's kernel ended
+    writes = 8.0 * units - residue
+    detail = {"dram_read_bytes": reads, "dram_write_bytes": writes, "l2_write_residue_bytes": residue,
+              "how": "ncu capture at 16 x 8,388,608: reads scaled by columns; writes = algorithmic minus the "
+                     "unscaled residue left in L2 at kernel end"}
+    return detail, reads + writes
 
 
 def measured_peak():
@@ -97,7 +114,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -300,6 +317,49 @@ def graph_seconds_per_call(step_fn, reset_fn, torch, stream, calls=40, replays=1
     return e0.elapsed_time(e1) * 1e-3 / (calls * replays)
 
 
+def build_topology(B, inputs, name):
+    w = inputs.WORKLOADS[name]
+    if w.topology == "er_mh":
+        adj, _ = inputs.er_adjacency(w.n, w.er_p, inputs.seed_for(name, inputs.P_GRAPH))
+        rowptr, col = inputs.adjacency_to_lists(adj)
+        return B.topology_build(B.CSR_MH, w.n, rowptr, col)
+    return B.topology_build({"ring": B.RING, "static_exp": B.STATIC_EXP, "one_peer_exp": B.ONE_PEER_EXP}[w.topology], w.n)
+
+
+def side_workload(name, B, inputs, torch, dev, stream, peak, steps=20, repeats=5):
+    """DecentLaM on another full-size workload: `repeats` timings of `steps` steps each (CUDA events, median and
+    best), its own clock samples, state freed on return."""
+    w = inputs.WORKLOADS[name]
+    gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    topo = build_topology(B, inputs, name)
+    x0 = inputs.normal_torch((w.n, w.d), w.x0_std, inputs.seed_for(name, inputs.P_X0), dev)
+    x = torch.empty_like(x0); m = torch.empty_like(x0)
+    g = inputs.normal_torch((w.n, w.d), w.g_std, inputs.seed_for(name, inputs.P_G0), dev, dtype=gdt)
+
+    def reset():
+        x.copy_(x0); m.zero_()
+
+    def step(k):
+        B.decentlam_step(topo, k, x, m, g, w.beta, w.gamma)
+
+    sampler = ClockSampler(dev.index or 0)
+    torch.cuda.synchronize()
+    sampler.start()
+    per_step = sorted(time_steps(step, reset, steps, 3, torch, stream)[0] / steps * 1e3 for _ in range(repeats))
+    clocks = sampler.stop()
+    err = B.kernel_error()
+    if err:
+        raise SystemExit(f"bench.py: step kernel reported error {err} on {name}")
+    bytes_alg = (16 + g.element_size()) * w.n * w.d
+    med = per_step[len(per_step) // 2]
+    del x, m, g, x0
+    torch.cuda.empty_cache()
+    return {"n": w.n, "d": w.d, "topology": w.topology, "g_dtype": w.g_dtype, "steps_each": steps, "repeats": repeats,
+            "ms_per_step": med, "ms_per_step_min": per_step[0], "value": w.n * w.d / (med * 1e-3), "unit": UNIT,
+            "gbs": bytes_alg / (med * 1e-3) / 1e9, "frac": bytes_alg / (med * 1e-3) / 1e9 / peak,
+            "algorithmic_bytes_per_launch": bytes_alg, "clocks": clocks}
+
+
 def run_ours(args):
     import torch
 
@@ -324,12 +384,7 @@ def run_ours(args):
     n, d = w.n, (args.columns or w.d)
     gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
 
-    if w.topology == "er_mh":
-        adj, _ = inputs.er_adjacency(n, w.er_p, inputs.seed_for(args.workload, inputs.P_GRAPH))
-        rowptr, col = inputs.adjacency_to_lists(adj)
-        topo = B.topology_build(B.CSR_MH, n, rowptr, col)
-    else:
-        topo = B.topology_build({"ring": B.RING, "static_exp": B.STATIC_EXP, "one_peer_exp": B.ONE_PEER_EXP}[w.topology], n)
+    topo = build_topology(B, inputs, args.workload)
 
     x0 = inputs.normal_torch((n, d), w.x0_std, inputs.seed_for(args.workload, inputs.P_X0) + rank, dev)
     x = torch.empty_like(x0); m = torch.empty_like(x0)
@@ -342,7 +397,8 @@ def run_ours(args):
     def decentlam(k):
         B.decentlam_step(topo, k, x, m, g, w.beta, w.gamma)
 
-    bytes_per_np = 16 + g.element_size()          # x, m read + x, m written + g read
+    g_esz = g.element_size()
+    bytes_per_np = 16 + g_esz                     # x, m read + x, m written + g read
     sampler = ClockSampler(local)
     if dist is not None:
         dist.barrier()
@@ -350,7 +406,15 @@ def run_ours(args):
     sampler.start()
     secs, launches = time_steps(decentlam, reset, args.steps, args.warmup, torch, stream, B.launch_count)
     torch.cuda.synchronize()
+    # spread of the same measurement: ten more repeats of 20 steps each (median and best); the clock sampler
+    # keeps running through them, so that even a short --steps run is covered by several samples
+    repeats = None
+    if world == 1 and not args.no_extra:
+        per_step = sorted(time_steps(decentlam, reset, 20, 3, torch, stream)[0] / 20 * 1e3 for _ in range(10))
+        repeats = {"steps_each": 20, "count": 10, "ms_per_step_median": per_step[5], "ms_per_step_min": per_step[0]}
     clocks = sampler.stop()
+    if clocks.get("sm_mhz"):
+        clocks["ms_per_step_x_sm_mhz"] = secs / args.steps * 1e3 * clocks["sm_mhz"]
     if dist is not None:
         dist.barrier()
     err = B.kernel_error()
@@ -360,11 +424,6 @@ def run_ours(args):
     value = job_units / job_secs
     peak, peak_kind = measured_peak()
     achieved = bytes_per_np * n * d * args.steps / secs / 1e9
-    # spread of the same measurement: five more repeats of 20 steps each (median and best)
-    repeats = None
-    if world == 1 and not args.no_extra:
-        per_step = sorted(time_steps(decentlam, reset, 20, 3, torch, stream)[0] / 20 * 1e3 for _ in range(5))
-        repeats = {"steps_each": 20, "count": 5, "ms_per_step_median": per_step[2], "ms_per_step_min": per_step[0]}
     # latency-bound sizes: the host's per-call issue time (about 10 us from Python) exceeds the kernel,
     # so the device-side figure comes from a replayed CUDA graph of 40 steps
     graph_us = None
@@ -436,6 +495,14 @@ def run_ours(args):
         oracle_build.build()
         cpu_baseline, _, _ = oracle_sample(args.workload)
 
+    # the other full-size workloads of the step, timed the same way in this run (the headline stays args.workload)
+    others = None
+    if world == 1 and not args.no_extra and not args.columns and args.workload == "cfg2":
+        del x, m, g, x0
+        torch.cuda.empty_cache()
+        others = {name: side_workload(name, B, inputs, torch, dev, stream, peak) for name in ("cfg3", "cfg5")}
+
+    traffic_detail, traffic_total = ncu_traffic(args.workload, n * d) if not args.columns else (None, None)
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -443,14 +510,120 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else ""), "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
                        "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
-                       "l2": f"working set {(8 + g.element_size()) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
+                       "l2": f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": ncu_traffic(args.workload, n * d), "peak_kind": f"of {peak_kind}",
+                         "traffic": traffic_total, "traffic_detail": traffic_detail, "peak_kind": f"of {peak_kind}",
                          "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d,
                          "copy_gbs_this_run": copy_gbs},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "cpu_baseline": cpu_baseline,
             "other_rules": extra, "repeats": repeats, "us_per_step_cuda_graph": graph_us,
+            "other_workloads": others,
         }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_sharded(args):
+    """Node-sharded DecentLaM step: every rank owns a block of rows, receives its halo (x and g rows of remote
+    neighbours), then runs the local kernel.  N > 1: one rank per GPU, halo exchange by NCCL send/recv, time =
+    max over ranks (exchange + kernel per step).  N = 1: rank 0's share of a `--sharded G` partition on this
+    GPU; the halo rows are copied from a second device buffer (standing in for the link) before every step."""
+    import torch
+
+    from paper_2104_11981_b200 import build as lib_build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        lib_build.build()
+    else:
+        t_wait = time.time()
+        while lib_build._stale() and time.time() - t_wait < 300:
+            time.sleep(1.0)
+    from paper_2104_11981_b200 import binding as B
+    from paper_2104_11981_b200 import exchange, inputs
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    args.warmup = max(args.warmup, 3)
+    rank, world, local, dist = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w = inputs.WORKLOADS[args.workload]
+    ranks = world if world > 1 else args.sharded
+    n, d = w.n, (args.columns or w.d)
+    gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    topo = build_topology(B, inputs, args.workload)
+    shard = B.topology_shard(topo, rank if world > 1 else 0, ranks)
+    lo, hi, max_halo = shard.rows
+    n_loc = hi - lo
+    x0 = inputs.normal_torch((n_loc, d), w.x0_std, inputs.seed_for(args.workload, inputs.P_X0) + rank, dev)
+    x = torch.empty_like(x0); m = torch.empty_like(x0)
+    g = inputs.normal_torch((n_loc, d), w.g_std, inputs.seed_for(args.workload, inputs.P_G0) + rank, dev, dtype=gdt)
+    halo_x = torch.zeros((max(1, max_halo), d), device=dev)
+    halo_g = torch.zeros((max(1, max_halo), d), device=dev, dtype=gdt)
+    # N = 1: "remote" rows live in a second buffer on this device
+    far_x = inputs.normal_torch((max(1, max_halo), d), w.x0_std, 7, dev) if world == 1 else None
+    far_g = inputs.normal_torch((max(1, max_halo), d), w.g_std, 8, dev, dtype=gdt) if world == 1 else None
+    stream = torch.cuda.current_stream()
+    period = topo.period
+    halo_counts = [len(shard.halo(s)[0]) for s in range(period)]
+    link_bytes = [c * d * (4 + g.element_size()) for c in halo_counts]
+
+    def reset():
+        x.copy_(x0); m.zero_()
+
+    def fill_halo(k):
+        h = halo_counts[k % period]
+        if world > 1:
+            exchange.post_halo_exchange(dist, shard, k % period, [x, g], [halo_x, halo_g])
+        elif h:
+            halo_x[:h].copy_(far_x[:h], non_blocking=True)
+            halo_g[:h].copy_(far_g[:h], non_blocking=True)
+
+    def kernel_only(k):
+        B.decentlam_step_sharded(shard, k, x, m, g, halo_x, halo_g, w.beta, w.gamma)
+
+    def full_step(k):
+        fill_halo(k)
+        kernel_only(k)
+
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    secs, launches = time_steps(full_step, reset, args.steps, args.warmup, torch, stream, B.launch_count)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ksecs, _ = time_steps(kernel_only, reset, args.steps, 3, torch, stream)
+    if dist is not None:
+        dist.barrier()
+    err = B.kernel_error()
+    if err:
+        raise SystemExit(f"bench.py: step kernel reported error {err}")
+    # whole job: all n rows advance one step per step (strong scaling: the same n x d state over more GPUs)
+    job_secs, _ = aggregate_over_ranks(dist, secs, 0, dev)
+    kjob_secs, _ = aggregate_over_ranks(dist, ksecs, 0, dev)
+    units_per_step = n * d if world > 1 else n_loc * d
+    peak, peak_kind = measured_peak()
+    mean_halo = sum(halo_counts) / period
+    local_bytes = (16 + g.element_size()) * n_loc * d + (4 + g.element_size()) * mean_halo * d   # own rows 3R+2W, halo rows read
+    if rank == 0:
+        line = {"metric": METRIC, "value": units_per_step * args.steps / job_secs, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3,
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": args.workload, "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
+                           "parallelism": f"node-sharded over {ranks} ranks" + ("" if world > 1 else
+                                          " (one GPU: rank 0's share, device copies stand in for the link)"),
+                           "rows_per_rank": n_loc, "halo_rows_per_slot": halo_counts,
+                           "l2": "inputs larger than the 126 MB L2; no flush"},
+                "roofline": {"bound": "hbm", "achieved": local_bytes * args.steps / ksecs / 1e9, "peak": peak, "unit": "GB/s",
+                             "frac": local_bytes * args.steps / ksecs / 1e9 / peak, "traffic": None,
+                             "peak_kind": f"of {peak_kind}", "kernel": "step_halo_kernel<decentlam>",
+                             "algorithmic_bytes_per_launch": local_bytes, "ms_per_kernel": kjob_secs / args.steps * 1e3},
+                "link": {"bytes_received_per_step_per_rank": link_bytes, "mean": sum(link_bytes) / period,
+                         "ms_at_770_GBs_model": sum(link_bytes) / period / 770e9 * 1e3,
+                         "note": "x and g rows of the remote neighbours (two arrays: see the header on accuracy)"},
+                "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "cpu_baseline": None}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
@@ -529,6 +702,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sharded:
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -219,6 +219,92 @@ DLM_API int pmsgd_step(int n, int64_t d, int64_t ld, float* x, float* m, const v
                int64_t ldg, float beta, float gamma, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------
+ * Row-sharded runs: the deployment the paper describes (Sec. 5 "Efficient implementation" and the
+ * workflow figure after Algorithm 2; Sec. 7 "Implementation").  Every GPU ("rank") holds a block of
+ * consecutive nodes, rank r of G the rows [r n / G, (r+1) n / G) (integer division) of x, m and g.
+ * Before a rank can update its rows it needs the rows of those neighbours that live on other ranks: its
+ * HALO for the iteration's time slot.  The library computes the exchange plan and runs the local
+ * update; moving the rows between GPUs is the caller's (peer copies, NCCL send/recv, ...), and the
+ * received rows always sit in a staging buffer in the rank's own memory before the kernel runs.
+ *
+ * What is exchanged.  DecentLaM (Algorithm 2) needs x_j and g_j of every remote neighbour j: two
+ * arrays.  The paper ships the single array x_j - gamma g_j and forms g~_i = (x_i - sum_j w_ij (x_j -
+ * gamma g_j)) / gamma from it; in fp32 that difference of nearly equal numbers loses eps |x| / gamma of
+ * absolute accuracy in m, about 1e-5 relative near consensus, so this library keeps the two operands
+ * apart (Eq. decentLaM-x-1 in difference form) at the price of twice the bytes on the link (1.5 times
+ * with bf16 gradients).  DmSGD (Algorithm 1) exchanges y_j = x_j - gamma m_j(new): one array, after the
+ * local momentum update, which is why it is two calls here with the exchange in between.
+ *
+ * G sharded calls (one per rank, each on its own rows and halo) give bitwise the result of one
+ * decentlam_step / dmsgd_step on the stacked state, when the latter takes its plain mixing loop
+ * (see dlm_set_tuning knob 7; the merged-staging kernel rounds differently).
+ * ------------------------------------------------------------------------------------ */
+typedef struct dlm_shard dlm_shard;
+
+/*
+ * Rank `rank` of `ranks`'s share of a topology: row range, exchange plan of every slot, local
+ * neighbour tables (uploaded to the current device, if there is one; without a CUDA device the
+ * handle is host-only: the plan can be read, steps fail with DLM_ERR_CUDA).  1 <= ranks <= n.
+ * The handle does not refer to `topo` afterwards.  Free with topology_shard_destroy (NULL accepted).
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE (rank or ranks out of range), DLM_ERR_CUDA.
+ */
+DLM_API int topology_shard(const dlm_topology* topo, int rank, int ranks, dlm_shard** out);
+DLM_API int topology_shard_destroy(dlm_shard* shard);
+
+/* Rows [*row_begin, *row_end) owned by the shard's rank, and the largest halo (rows) over all slots:
+ * the number of rows a halo staging buffer must hold.  Any out-pointer may be NULL. */
+DLM_API int topology_shard_rows(const dlm_shard* shard, int* row_begin, int* row_end, int* max_halo);
+
+/*
+ * Receive side of the exchange plan for one slot: the *count remote rows this rank needs, as global
+ * row indices in ascending order (rows[t] must end up in row t of the halo buffers), and the rank
+ * that owns each (owners[t]).  Borrowed host pointers, valid until topology_shard_destroy; any
+ * out-pointer may be NULL.  Errors: DLM_ERR_NULL, DLM_ERR_SHAPE (slot outside [0, period)).
+ */
+DLM_API int topology_halo(const dlm_shard* shard, int slot, const int32_t** rows, const int32_t** owners, int* count);
+
+/*
+ * Send side: the *count rows owned by this rank that rank `peer` needs in this slot (global indices,
+ * ascending) and the row of peer's halo buffers each one goes to (dst_slots[t]).  The plans of all
+ * ranks agree: what r sends to r' is exactly what r' expects from r.  peer == own rank gives count 0.
+ */
+DLM_API int topology_halo_sends(const dlm_shard* shard, int slot, int peer, const int32_t** rows,
+                                const int32_t** dst_slots, int* count);
+
+/*
+ * DecentLaM step of one rank (Eqs. decentLaM-x-1..3 restricted to the rank's rows).
+ *   x, m, g     : device, the rank's OWN rows [n_loc, d] (n_loc = row_end - row_begin), as in decentlam_step;
+ *                 x and m updated in place
+ *   halo_x      : device fp32 [halo, d], row stride ld_halo_x: row t = x of node rows[t] of topology_halo
+ *                 for slot k mod period, as it was BEFORE this iteration on its owner
+ *   halo_g      : device [halo, d] of g's dtype, row stride ld_halo_g: the same nodes' gradients
+ *                 (both may be NULL when the slot's halo is empty)
+ * The kernel stages its tiles with 2-D bulk copies: every base pointer 16-byte aligned, every row
+ * stride a multiple of 16 bytes (DLM_ERR_ALIGN otherwise); d itself is arbitrary.  At most 256 own rows
+ * and 256 halo rows per rank (DLM_ERR_UNSUPPORTED beyond).  Traffic per own node-parameter: 20 bytes
+ * (18 with bf16 g) plus 8 (6) bytes per halo node-parameter read.
+ * Errors: DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_ALIGN, DLM_ERR_ALIAS (x or m overlapping any other
+ * buffer), DLM_ERR_HYPER, DLM_ERR_KIND, DLM_ERR_UNSUPPORTED, DLM_ERR_CUDA.
+ */
+DLM_API int decentlam_step_sharded(const dlm_shard* shard, int64_t k, int64_t d, int64_t ld, float* x, float* m,
+                                   const void* g, int g_dtype, int64_t ldg, const float* halo_x, int64_t ld_halo_x,
+                                   const void* halo_g, int64_t ld_halo_g, float beta, float gamma, void* cuda_stream);
+
+/*
+ * DmSGD of one rank in two calls (Algorithm 1), the exchange of y between them:
+ *   dmsgd_local_sharded      m_i <- beta m_i + g_i ;  x_i <- y_i = x_i - gamma m_i(new)   on the own rows
+ *                            (any alignment; no topology involved beyond the row count)
+ *   -- the caller sends its y rows and receives the neighbours' into halo_x --
+ *   partial_average_sharded  x_i <- x_i + sum_{j in N_i, j != i} w_ij (x_j - x_i)          (Eq. partial-ave)
+ *                            own rows of x in place, halo_x as for decentlam_step_sharded
+ * Alignment, size limits and errors of partial_average_sharded as for decentlam_step_sharded.
+ */
+DLM_API int dmsgd_local_sharded(const dlm_shard* shard, int64_t d, int64_t ld, float* x, float* m, const void* g,
+                                int g_dtype, int64_t ldg, float beta, float gamma, void* cuda_stream);
+DLM_API int partial_average_sharded(const dlm_shard* shard, int64_t k, int64_t d, int64_t ld, float* x,
+                                    const float* halo_x, int64_t ld_halo_x, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------
  * Full-batch least-squares gradient of the linear-regression experiment (App. G):
  *   f_i(x) = (scale/2) ||A_i x - b_i||^2 ,   g_i = scale * A_i^T (A_i x_i - b_i).
  *   A : device fp32 [n, p, q] row-major, 16-byte aligned; 1 <= q <= 8192, n <= DLM_LSQ_MAX_NODES
@@ -298,8 +384,10 @@ DLM_API int lsq_grad_gram(int n, int q, const float* H, const float* c, const fl
 DLM_API int64_t dlm_launch_count(void);
 
 /*
- * The pipelined step kernel bounds every wait on its copy barriers; if a wait ever runs out the
- * kernel records a non-zero code, stops early and the step's output is incomplete.  This call
+ * The kernels that stage their tiles with bulk copies bound every wait on a copy barrier; if a wait
+ * ever runs out the kernel records a non-zero code and stops early, and the call that launched it has
+ * still returned DLM_OK (it only enqueues).  The outputs of every step and gradient call issued since
+ * the last check are therefore to be trusted only once this function has returned 0 in *flag.  It
  * synchronises with the device, returns the recorded code in *flag (0 = none) and clears it.
  */
 DLM_API int dlm_kernel_error(int* flag);
@@ -315,13 +403,14 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 5  neighbour tables: 1 = staged in shared memory, 2 = read from global memory
  *   knob 6  threads per CTA of the pipeline kernels (128, 256 or 512)
  *   knob 7  1 = pipeline kernel with the plain mixing loop, 2 = merged-staging kernel (one staged
- *           value per neighbour)
+ *           value per neighbour), 3 = its compact-table form for decentlam_step where the graph allows it
  *   knob 8  lsq_grad and lsq_grad_gram: row chunks per node (at most 64)
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
  *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
  *   knob 11 lsq_grad_gram: share of H kept in L2 with evict-last priority between calls, in 1/1000
  *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
  *           size, else none)
+ *   knob 12 block size of the compact-table merged kernel (256, 384 or 512)
  * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
  * the default on long rows: 12 or more entries, 8 or more for dmsgd_step and up to 128 nodes) arranges the same sum differently and
  * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.

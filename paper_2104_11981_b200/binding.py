@@ -55,6 +55,15 @@ for _name in ("decentlam_step", "dmsgd_step"):
 _lib.decentlam_step_host_gradients.argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _vp, _i64, _flt,
                                                _flt, _vp]
 _lib.dsgd_step.argtypes = [_vp, _i64, _int, _i64, _i64, _vp, _vp, _int, _i64, _flt, _int, _vp]
+_lib.topology_shard.argtypes = [_vp, _int, _int, ctypes.POINTER(_vp)]
+_lib.topology_shard_destroy.argtypes = [_vp]
+_lib.topology_shard_rows.argtypes = [_vp, ctypes.POINTER(_int), ctypes.POINTER(_int), ctypes.POINTER(_int)]
+_lib.topology_halo.argtypes = [_vp, _int, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_int)]
+_lib.topology_halo_sends.argtypes = [_vp, _int, _int, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_int)]
+_lib.decentlam_step_sharded.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _int, _i64, _vp, _i64, _vp, _i64, _flt, _flt,
+                                        _vp]
+_lib.dmsgd_local_sharded.argtypes = [_vp, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
+_lib.partial_average_sharded.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp]
 _lib.pmsgd_step.argtypes = [_int, _i64, _i64, _vp, _vp, _vp, _int, _i64, _flt, _flt, _vp]
 _lib.lsq_grad_workspace_bytes.argtypes = [_int, _int, _int]
 _lib.lsq_grad_workspace_bytes.restype = _i64
@@ -69,6 +78,8 @@ _lib.dlm_set_tuning.argtypes = [_int, _int]
 
 EXPORTS = ["dlm_status_string", "topology_build", "topology_build_periodic", "topology_period", "topology_nodes", "topology_tables_host",
            "topology_tables_device", "topology_destroy", "decentlam_step", "decentlam_step_host_gradients", "dmsgd_step", "dsgd_step", "pmsgd_step",
+           "topology_shard", "topology_shard_destroy", "topology_shard_rows", "topology_halo", "topology_halo_sends",
+           "decentlam_step_sharded", "dmsgd_local_sharded", "partial_average_sharded",
            "lsq_grad_workspace_bytes", "lsq_grad", "lsq_grad_static", "lsq_gram_build", "lsq_grad_gram", "dlm_launch_count", "dlm_kernel_error", "dlm_set_tuning"]
 
 
@@ -222,6 +233,93 @@ def dsgd_step(topo, k, x, g, gamma, variant=DSGD_ATC, stream=None):
     n, d = x.shape
     _check(_lib.dsgd_step(topo.handle, k, n, d, x.stride(0), _vp(x.data_ptr()), _vp(g.data_ptr()), gd, g.stride(0),
                           gamma, variant, _stream_ptr(stream)), "dsgd_step")
+
+
+class Shard:
+    """Owner of a dlm_shard handle: one rank's share of a topology in a row-sharded run."""
+
+    def __init__(self, handle, period):
+        self.handle = handle
+        self.period = period
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def destroy(self):
+        if getattr(self, "handle", None):
+            _lib.topology_shard_destroy(self.handle)
+            self.handle = None
+
+    @property
+    def rows(self):
+        """(row_begin, row_end, max_halo)."""
+        lo, hi, mh = _int(), _int(), _int()
+        _check(_lib.topology_shard_rows(self.handle, ctypes.byref(lo), ctypes.byref(hi), ctypes.byref(mh)),
+               "topology_shard_rows")
+        return lo.value, hi.value, mh.value
+
+    @staticmethod
+    def _pair(pa, pb, count):
+        import numpy as np
+        if count == 0:
+            return np.zeros(0, np.int32), np.zeros(0, np.int32)
+        a = np.ctypeslib.as_array(ctypes.cast(pa, _i32p), shape=(count,)).copy()
+        b = np.ctypeslib.as_array(ctypes.cast(pb, _i32p), shape=(count,)).copy()
+        return a, b
+
+    def halo(self, slot):
+        """(rows, owners): the remote rows this rank receives in `slot` (ascending global indices; rows[t]
+        goes to row t of the halo buffers) and the rank owning each."""
+        pr, po, c = _vp(), _vp(), _int()
+        _check(_lib.topology_halo(self.handle, slot, ctypes.byref(pr), ctypes.byref(po), ctypes.byref(c)), "topology_halo")
+        return self._pair(pr, po, c.value)
+
+    def sends(self, slot, peer):
+        """(rows, dst_slots): own rows (global indices) that `peer` needs in `slot`, and the halo row of
+        the peer each one lands in."""
+        pr, pd, c = _vp(), _vp(), _int()
+        _check(_lib.topology_halo_sends(self.handle, slot, peer, ctypes.byref(pr), ctypes.byref(pd), ctypes.byref(c)),
+               "topology_halo_sends")
+        return self._pair(pr, pd, c.value)
+
+
+def topology_shard(topo, rank, ranks):
+    out = _vp()
+    _check(_lib.topology_shard(topo.handle, rank, ranks, ctypes.byref(out)), "topology_shard")
+    return Shard(out, topo.period)
+
+
+def _halo_ptr(t):
+    return (_vp(t.data_ptr()), t.stride(0)) if t is not None and t.numel() > 0 else (None, 0)
+
+
+def decentlam_step_sharded(shard, k, x, m, g, halo_x, halo_g, beta, gamma, stream=None):
+    """DecentLaM step of one rank: x, m, g are the rank's own rows [n_loc, d]; halo_x, halo_g [halo, d] hold
+    the remote neighbours' rows in the order of shard.halo(k % period) (None when the halo is empty)."""
+    n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
+    (phx, ldhx), (phg, ldhg) = _halo_ptr(halo_x), _halo_ptr(halo_g)
+    _check(_lib.decentlam_step_sharded(shard.handle, k, d, ld, px, pm, pg, gd, ldg, phx, ldhx, phg, ldhg, beta, gamma,
+                                       _stream_ptr(stream)), "decentlam_step_sharded")
+
+
+def dmsgd_local_sharded(shard, x, m, g, beta, gamma, stream=None):
+    """First half of a sharded DmSGD step on the rank's own rows: m <- beta m + g, x <- x - gamma m."""
+    n, d, ld, px, pm, pg, gd, ldg = _state_args(x, m, g)
+    _check(_lib.dmsgd_local_sharded(shard.handle, d, ld, px, pm, pg, gd, ldg, beta, gamma, _stream_ptr(stream)),
+           "dmsgd_local_sharded")
+
+
+def partial_average_sharded(shard, k, x, halo_x, stream=None):
+    """Second half: x_i <- x_i + sum_{j != i} w_ij (x_j - x_i) over own rows, remote rows from halo_x."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+    n, d = x.shape
+    phx, ldhx = _halo_ptr(halo_x)
+    _check(_lib.partial_average_sharded(shard.handle, k, d, x.stride(0), _vp(x.data_ptr()), phx, ldhx,
+                                        _stream_ptr(stream)), "partial_average_sharded")
 
 
 def pmsgd_step(x, m, g, beta, gamma, stream=None):

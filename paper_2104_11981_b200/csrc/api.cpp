@@ -84,6 +84,10 @@ int topo_step(int rule, const dlm_topology* topo, int64_t k, int n, int64_t d, i
     a.rows = s.d_rows;
     a.ent = s.d_ent;
     a.selfw = s.d_selfw;
+    a.compact = s.d_compact;
+    a.compact_bytes = (int)s.compact.size();
+    a.compact_nw = s.compact_nw;
+    a.compact_noff = s.compact_noff;
     a.nnz = (int)s.col.size();
     a.max_degree = s.max_degree;
     a.beta = beta;
@@ -236,7 +240,9 @@ int lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x
     if (overlap(rg, ra) || overlap(rg, rb) || overlap(rg, rx) || overlap(rw, ra) || overlap(rw, rb) ||
         overlap(rw, rx) || overlap(rw, rg))
         return DLM_ERR_ALIAS;
-    return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, reinterpret_cast<float*>(workspace), cuda_stream);
+    const int S = dlm_lsq_splits(n, p, q);  // at most the 64 splits the workspace size is checked against
+    if (S < 1) return DLM_ERR_CUDA;
+    return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, reinterpret_cast<float*>(workspace), S, cuda_stream);
 }
 
 int lsq_gram_build(int n, int p, int q, const float* A, const float* b, float scale, float* H, float* c,
@@ -270,18 +276,21 @@ int dlm_set_tuning(int knob, int value) {
     case 9: g_lsq_tune_bulk = value; return DLM_OK;
     case 10: g_pmsgd_tune_cap = value; return DLM_OK;
     case 11: g_l2_keep_permille = value; return DLM_OK;
+    case 12: return dlm_compact_set_threads(value);
     default: return DLM_ERR_KIND;
     }
 }
 
 int dlm_kernel_error(int* flag) {
     if (!flag) return DLM_ERR_NULL;
-    int step = 0, lsq = 0;
+    int step = 0, lsq = 0, shard = 0;
     int rc = dlm_step_take_error(&step);
     if (rc != DLM_OK) return rc;
     rc = dlm_lsq_take_error(&lsq);
     if (rc != DLM_OK) return rc;
-    *flag = step != 0 ? step : lsq;
+    rc = dlm_shard_take_error(&shard);
+    if (rc != DLM_OK) return rc;
+    *flag = step != 0 ? step : lsq != 0 ? lsq : shard;
     return DLM_OK;
 }
 

@@ -12,9 +12,13 @@
 #include <algorithm>
 #include <cstdint>
 
+#include "dlm_device.cuh"
 #include "dlm_internal.h"
 
 namespace {
+
+using dlm::mbar_wait;
+using dlm::smem_u32;
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
@@ -96,23 +100,7 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_rows_kernel(int p, int q
 // chunk.  Summation order per row and per column is that of lsq_partial_rows_kernel, so both
 // give bitwise the same partial sums.
 constexpr int kStages = 3;
-constexpr uint32_t kLsqWaitLimit = 1u << 22;
-__device__ int g_lsq_kernel_error = 0;
-
-__device__ __forceinline__ uint32_t lsq_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool lsq_mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kLsqWaitLimit; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if (i > 32) __nanosleep(64);
-    }
-    return false;
-}
+__device__ int g_lsq_kernel_error = 0;  // set to a non-zero code if a bounded wait ran out
 
 // L2 policy for the bulk copies of a matrix that every iteration reads again (H of the Gram form):
 // the given fraction of its lines is kept with evict-last priority so that it is still cached at the
@@ -144,7 +132,7 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
     extern __shared__ __align__(16) unsigned char lsq_smem[];
     // launched with programmatic stream serialization: x comes from the kernel before this one
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    unsigned char* base = lsq_smem + ((128u - (lsq_smem_u32(lsq_smem) & 127u)) & 127u);
+    unsigned char* base = lsq_smem + ((128u - (smem_u32(lsq_smem) & 127u)) & 127u);
     const uint32_t chunk_bytes = (uint32_t)kWarps * q * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)kStages * chunk_bytes);
     const int s = blockIdx.x, i = blockIdx.y;
@@ -158,13 +146,13 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
     auto issue = [&](int st, int c) {
         const int row = r0 + c * kWarps;
         const uint32_t bytes = (uint32_t)min(kWarps, r1 - row) * q * 4;
-        const uint32_t bar = lsq_smem_u32(&bars[st]);
+        const uint32_t bar = smem_u32(&bars[st]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        bulk_copy(lsq_smem_u32(base + (size_t)st * chunk_bytes), Ai + (size_t)row * q, bytes, bar, false, 0);
+        bulk_copy(smem_u32(base + (size_t)st * chunk_bytes), Ai + (size_t)row * q, bytes, bar, false, 0);
     };
     if (threadIdx.x == 0) {
         for (int st = 0; st < kStages; ++st)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lsq_smem_u32(&bars[st])), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bars[st])), "r"(1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int st = 0; st < kStages && st < chunks; ++st) issue(st, st);
     }
@@ -179,12 +167,14 @@ __global__ void __launch_bounds__(kThreads) lsq_partial_bulk_kernel(int p, int q
         const int st = c % kStages;
         const int r = r0 + c * kWarps + warp;
         const float bv = r < r1 ? bi[r] : 0.f;  // in flight while the chunk lands
-        const bool arrived = lsq_mbar_wait(lsq_smem_u32(&bars[st]), (uint32_t)((c / kStages) & 1));
+        const bool arrived = mbar_wait(smem_u32(&bars[st]), (uint32_t)((c / kStages) & 1));
         if (!__syncthreads_and(arrived)) {
             if (threadIdx.x == 0) {
                 atomicExch(&g_lsq_kernel_error, 2);
-                for (int j = c + 1; j < chunks && j < c + kStages; ++j)
-                    lsq_mbar_wait(lsq_smem_u32(&bars[j % kStages]), (uint32_t)((j / kStages) & 1));
+                // every copy still on its way, the awaited one included, gets one more bounded wait
+                // before the CTA's shared memory is released
+                for (int j = c; j < chunks && j < c + kStages; ++j)
+                    mbar_wait(smem_u32(&bars[j % kStages]), (uint32_t)((j / kStages) & 1));
             }
             __syncthreads();
             return;
@@ -344,11 +334,12 @@ static float l2_keep_fraction(double bytes) {
     return (bytes <= room || bytes > 2.0 * (double)l2) ? 0.0f : (float)(room / bytes);
 }
 
+// S = row chunks per node (from dlm_lsq_splits, computed ONCE by the caller, who also sized or checked
+// the [n, S, q] scratch with that same value).
 int dlm_launch_lsq_grad(int n, int p, int q, const float* A, const float* b, const float* x, float* g,
-                        float scale, float* partial, void* stream) {
+                        float scale, float* partial, int S, void* stream) {
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    int S = dlm_lsq_splits(n, p, q);
-    if (S < 1) return DLM_ERR_CUDA;
+    if (S < 1 || S > kMaxSplits) return DLM_ERR_CUDA;
     int rows = ((p + S - 1) / S + kWarps - 1) / kWarps * kWarps;
     dim3 grid((unsigned)S, (unsigned)n);
     const bool fast = (q % 128 == 0) && q <= 1024;
@@ -467,7 +458,7 @@ extern "C" DLM_API int lsq_grad_static(int n, int p, int q, const float* A, cons
     if (rc != DLM_OK) return rc;
     // Every partial [i, s, :] that the reduction reads is written by the first kernel of this same
     // call, so nothing left over from an earlier call is ever consumed and nothing needs clearing.
-    return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, scratch, cuda_stream);
+    return dlm_launch_lsq_grad(n, p, q, A, b, x, g, scale, scratch, S, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -666,7 +657,7 @@ __global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int row
                                                                    float* __restrict__ g) {
     extern __shared__ __align__(16) unsigned char lsq_smem[];
     asm volatile("griddepcontrol.wait;" ::: "memory");  // x may come from the kernel before this one
-    unsigned char* base = lsq_smem + ((128u - (lsq_smem_u32(lsq_smem) & 127u)) & 127u);
+    unsigned char* base = lsq_smem + ((128u - (smem_u32(lsq_smem) & 127u)) & 127u);
     const uint32_t chunk_bytes = (uint32_t)kWarps * q * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)kStages * chunk_bytes);
     const int s = blockIdx.x, i = blockIdx.y;
@@ -683,13 +674,13 @@ __global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int row
     auto issue = [&](int st, int c) {
         const int row = r0 + c * kWarps;
         const uint32_t bytes = (uint32_t)min(kWarps, r1 - row) * q * 4;
-        const uint32_t bar = lsq_smem_u32(&bars[st]);
+        const uint32_t bar = smem_u32(&bars[st]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        bulk_copy(lsq_smem_u32(base + (size_t)st * chunk_bytes), Hi + (size_t)row * q, bytes, bar, hint, pol);
+        bulk_copy(smem_u32(base + (size_t)st * chunk_bytes), Hi + (size_t)row * q, bytes, bar, hint, pol);
     };
     if (threadIdx.x == 0) {
         for (int st = 0; st < kStages; ++st)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lsq_smem_u32(&bars[st])), "r"(1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&bars[st])), "r"(1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int st = 0; st < kStages && st < chunks; ++st) issue(st, st);
     }
@@ -701,12 +692,14 @@ __global__ void __launch_bounds__(kThreads) gram_grad_bulk_kernel(int q, int row
         const int st = c % kStages;
         const int r = r0 + c * kWarps + warp;
         const float cv = r < r1 ? ci[r] : 0.f;  // in flight while the chunk lands
-        const bool arrived = lsq_mbar_wait(lsq_smem_u32(&bars[st]), (uint32_t)((c / kStages) & 1));
+        const bool arrived = mbar_wait(smem_u32(&bars[st]), (uint32_t)((c / kStages) & 1));
         if (!__syncthreads_and(arrived)) {
             if (threadIdx.x == 0) {
                 atomicExch(&g_lsq_kernel_error, 3);
-                for (int j = c + 1; j < chunks && j < c + kStages; ++j)
-                    lsq_mbar_wait(lsq_smem_u32(&bars[j % kStages]), (uint32_t)((j / kStages) & 1));
+                // every copy still on its way, the awaited one included, gets one more bounded wait
+                // before the CTA's shared memory is released
+                for (int j = c; j < chunks && j < c + kStages; ++j)
+                    mbar_wait(smem_u32(&bars[j % kStages]), (uint32_t)((j / kStages) & 1));
             }
             __syncthreads();
             return;

@@ -8,6 +8,7 @@
 
 #include <cstdint>
 
+#include "dlm_device.cuh"
 #include "dlm_internal.h"
 
 int g_pmsgd_tune_cap = 0;  // blocks per SM of the grid, 0 = one block per 256 column groups
@@ -17,47 +18,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 8;
 
-template <int VEC>
-struct Pack {
-    float v[VEC];
-};
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_f32(const float* p);
-template <>
-__device__ __forceinline__ Pack<4> ld_f32<4>(const float* p) {
-    float4 t = *reinterpret_cast<const float4*>(p);
-    return {{t.x, t.y, t.z, t.w}};
-}
-template <>
-__device__ __forceinline__ Pack<1> ld_f32<1>(const float* p) {
-    return {{*p}};
-}
-template <int VEC>
-__device__ __forceinline__ void st_f32(float* p, const Pack<VEC>& a);
-template <>
-__device__ __forceinline__ void st_f32<4>(float* p, const Pack<4>& a) {
-    *reinterpret_cast<float4*>(p) = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
-}
-template <>
-__device__ __forceinline__ void st_f32<1>(float* p, const Pack<1>& a) {
-    *p = a.v[0];
-}
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_g(const float* p) {
-    return ld_f32<VEC>(p);
-}
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_g(const __nv_bfloat16* p);
-template <>
-__device__ __forceinline__ Pack<4> ld_g<4>(const __nv_bfloat16* p) {
-    uint2 u = *reinterpret_cast<const uint2*>(p);
-    return {{__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-             __uint_as_float(u.y & 0xffff0000u)}};
-}
-template <>
-__device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
-    return {{__uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short*>(p)) << 16)}};
-}
+using namespace dlm;
 
 // One pass over the columns [c, c + VEC) of all rows.
 template <typename GT, int VEC>

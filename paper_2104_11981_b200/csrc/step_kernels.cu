@@ -6,14 +6,14 @@
 // and only then writes x and m of the same tile.  This makes the in-place update exact
 // (simultaneous update of all nodes) with each of x, m, g read once and x, m written once.
 //
-// Three kernels:
+// Two kernels here, a third in step_merged.cu:
 //   step_tma_kernel     the tile arrives by 2-D tensor bulk copies (cp.async.bulk.tensor) completing on an
 //                       mbarrier; by default one stage per CTA and a grid of many short-lived CTAs, several
 //                       resident per SM (a persistent multi-stage pipeline is selectable).  Needs 16-byte
 //                       aligned rows; more than 256 nodes arrive as several row boxes per array.
 //   step_tile_kernel    plain vector/scalar loads into shared memory; any alignment, n up to 2048, also
 //                       used for tiny problems and for the last d mod 4 columns.
-//   step_merged_kernel  for long neighbour lists: one staged value per neighbour (see its own header).
+//   step_merged_kernel  for long neighbour lists: one staged value per neighbour (see its own file).
 // The first two call the same per-element update functions, so their results are bitwise identical; the
 // third evaluates the same sums in another arrangement and agrees with them to rounding.
 #include <cuda.h>
@@ -22,184 +22,30 @@
 
 #include <algorithm>
 #include <cstdint>
-#include <mutex>
 
+#include "dlm_device.cuh"
 #include "dlm_internal.h"
+#include "dlm_launch.h"
+
+int g_tune_path = 0;
+int g_tune_cols = 0;
+int g_tune_stages = 0;
+int g_tune_ctas = 0;
+int g_tune_threads = 0;
+int g_tune_mix = 0;
+int g_tune_tables = 0;
+int g_tune_tiles_per_cta = 0;
 
 namespace {
+
+using namespace dlm;
 
 constexpr int kThreads = 256;     // tile kernel block size
 constexpr int kMaxThreads = 512;  // pipeline kernel block size limit
 constexpr int kMaxStages = 8;
-constexpr uint32_t kWaitLimit = 1u << 22;  // polls before a pipeline wait gives up
 
 __device__ int g_kernel_error = 0;  // set to a non-zero code if a bounded wait ran out
 
-// ---------------------------------------------------------------------------------------------
-// Per-element arithmetic (fp32, explicit FMAs so every kernel variant rounds identically).
-// ---------------------------------------------------------------------------------------------
-// DecentLaM (Eqs. decentLaM-x-1..3):  g~ = (W g)_i + ((I - W) x)_i / gamma ; m' = beta m + g~ ; x' = x - gamma m'
-__device__ __forceinline__ void decentlam_finish(float mixg, float cons, float xi, float mi, float beta,
-                                                 float gamma, float inv_gamma, float& mn, float& xn) {
-    float gt = fmaf(cons, inv_gamma, mixg);
-    mn = fmaf(beta, mi, gt);
-    xn = fmaf(-gamma, mn, xi);
-}
-// DmSGD (Algorithm 1), local half:  m' = beta m + g ; y = x - gamma m'
-__device__ __forceinline__ void dmsgd_local(float xi, float mi, float gi, float beta, float gamma, float& mn,
-                                            float& y) {
-    mn = fmaf(beta, mi, gi);
-    y = fmaf(-gamma, mn, xi);
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
-
-template <int VEC>
-struct Pack {
-    float v[VEC];
-};
-
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_f32(const float* p);
-template <>
-__device__ __forceinline__ Pack<4> ld_f32<4>(const float* p) {
-    float4 t = *reinterpret_cast<const float4*>(p);
-    return {{t.x, t.y, t.z, t.w}};
-}
-template <>
-__device__ __forceinline__ Pack<1> ld_f32<1>(const float* p) {
-    return {{*p}};
-}
-template <int VEC>
-__device__ __forceinline__ void st_f32(float* p, const Pack<VEC>& a);
-template <>
-__device__ __forceinline__ void st_f32<4>(float* p, const Pack<4>& a) {
-    *reinterpret_cast<float4*>(p) = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
-}
-template <>
-__device__ __forceinline__ void st_f32<1>(float* p, const Pack<1>& a) {
-    *p = a.v[0];
-}
-// gradient loads: fp32 or bf16 bit patterns widened exactly
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_g(const float* p) {
-    return ld_f32<VEC>(p);
-}
-template <int VEC>
-__device__ __forceinline__ Pack<VEC> ld_g(const __nv_bfloat16* p);
-template <>
-__device__ __forceinline__ Pack<4> ld_g<4>(const __nv_bfloat16* p) {
-    uint2 u = *reinterpret_cast<const uint2*>(p);
-    return {{__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-             __uint_as_float(u.y & 0xffff0000u)}};
-}
-template <>
-__device__ __forceinline__ Pack<1> ld_g<1>(const __nv_bfloat16* p) {
-    return {{bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(p))}};
-}
-
-
-// Neighbour tables of the current slot, either copied to shared memory or left in global memory.
-// DecentLaM reads packed entries {column, bits of the weight}, one 64-bit load per neighbour (3.6 % on
-// the 64-node bf16 workload); the averaging rules read separate column and weight arrays, which keeps
-// the DSGD kernels at 40 registers, i.e. six CTAs per SM (with packed entries: 49 registers, 13 % slower).
-template <bool PACKED>
-struct Tables;
-template <>
-struct Tables<false> {
-    const int* rowptr;
-    const int* col;
-    const float* val;
-    const int* order;
-};
-template <>
-struct Tables<true> {
-    const int* rowptr;
-    const int2* ent;
-    const int* order;
-};
-
-// smem_tables must be 8-byte aligned.
-template <bool PACKED>
-__device__ __forceinline__ Tables<PACKED> stage_tables(const dlm_step_args& a, void* smem_tables, bool in_smem);
-template <>
-__device__ __forceinline__ Tables<false> stage_tables<false>(const dlm_step_args& a, void* smem_tables, bool in_smem) {
-    if (!in_smem) return {a.rowptr, a.col, a.val, a.order};
-    int* s_rowptr = reinterpret_cast<int*>(smem_tables);
-    int* s_order = s_rowptr + (a.n + 1);
-    int* s_col = s_order + a.n;
-    float* s_val = reinterpret_cast<float*>(s_col + a.nnz);
-    for (int i = threadIdx.x; i <= a.n; i += blockDim.x) s_rowptr[i] = a.rowptr[i];
-    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s_order[i] = a.order[i];
-    for (int i = threadIdx.x; i < a.nnz; i += blockDim.x) {
-        s_col[i] = a.col[i];
-        s_val[i] = a.val[i];
-    }
-    return {s_rowptr, s_col, s_val, s_order};
-}
-template <>
-__device__ __forceinline__ Tables<true> stage_tables<true>(const dlm_step_args& a, void* smem_tables, bool in_smem) {
-    const int2* ent = reinterpret_cast<const int2*>(a.ent);
-    if (!in_smem) return {a.rowptr, ent, a.order};
-    int2* s_ent = reinterpret_cast<int2*>(smem_tables);
-    int* s_rowptr = reinterpret_cast<int*>(s_ent + a.nnz);
-    int* s_order = s_rowptr + (a.n + 1);
-    for (int i = threadIdx.x; i <= a.n; i += blockDim.x) s_rowptr[i] = a.rowptr[i];
-    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s_order[i] = a.order[i];
-    for (int i = threadIdx.x; i < a.nnz; i += blockDim.x) s_ent[i] = ent[i];
-    return {s_rowptr, s_ent, s_order};
-}
-
-// Mix one item (row i, VEC consecutive columns at tile offset off) of the DecentLaM rule.
-//   xs, gs: staged tiles [n][C] (gs may hold bf16 when GS is __nv_bfloat16)
-template <int VEC, typename GS>
-__device__ __forceinline__ void decentlam_item(const Tables<true>& t, int i, int off, int C, const float* xs,
-                                               const GS* gs, const Pack<VEC>& mi, float beta, float gamma,
-                                               float inv_gamma, Pack<VEC>& mn, Pack<VEC>& xn) {
-    const Pack<VEC> xi = ld_f32<VEC>(xs + i * C + off);
-    float mixg[VEC], cons[VEC];
-#pragma unroll
-    for (int u = 0; u < VEC; ++u) mixg[u] = cons[u] = 0.0f;
-    const int p1 = t.rowptr[i + 1];
-    for (int p = t.rowptr[i]; p < p1; ++p) {  // neighbours in ascending order
-        const int2 en = t.ent[p];
-        const int j = en.x;
-        const float w = __int_as_float(en.y);
-        const Pack<VEC> gj = ld_g<VEC>(gs + j * C + off);
-#pragma unroll
-        for (int u = 0; u < VEC; ++u) mixg[u] = fmaf(w, gj.v[u], mixg[u]);
-        if (j != i) {
-            const Pack<VEC> xj = ld_f32<VEC>(xs + j * C + off);
-#pragma unroll
-            for (int u = 0; u < VEC; ++u) cons[u] = fmaf(w, xi.v[u] - xj.v[u], cons[u]);
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < VEC; ++u)
-        decentlam_finish(mixg[u], cons[u], xi.v[u], mi.v[u], beta, gamma, inv_gamma, mn.v[u], xn.v[u]);
-}
-
-// Partial average of the DmSGD rule on staged y = x - gamma m':  x' = y_i + sum_{j != i} w_ij (y_j - y_i)
-template <int VEC>
-__device__ __forceinline__ void dmsgd_item(const Tables<false>& t, int i, int off, int C, const float* ys,
-                                           Pack<VEC>& xn) {
-    const Pack<VEC> yi = ld_f32<VEC>(ys + i * C + off);
-    float acc[VEC];
-#pragma unroll
-    for (int u = 0; u < VEC; ++u) acc[u] = 0.0f;
-    const int p1 = t.rowptr[i + 1];
-    for (int p = t.rowptr[i]; p < p1; ++p) {
-        const int j = t.col[p];
-        if (j == i) continue;
-        const float w = t.val[p];
-        const Pack<VEC> yj = ld_f32<VEC>(ys + j * C + off);
-#pragma unroll
-        for (int u = 0; u < VEC; ++u) acc[u] = fmaf(w, yj.v[u] - yi.v[u], acc[u]);
-    }
-#pragma unroll
-    for (int u = 0; u < VEC; ++u) xn.v[u] = yi.v[u] + acc[u];
-}
 
 // ---------------------------------------------------------------------------------------------
 // Plain-load tile kernel (any alignment).  C is a power of two multiple of VEC.
@@ -282,50 +128,6 @@ __global__ void __launch_bounds__(kThreads) step_tile_kernel(dlm_step_args a, in
 // Shared memory per stage: x tile [n][C] fp32 | m tile [n][C] fp32 | g tile [n][C] GT, each
 // rounded up to 128 bytes; then `stages` mbarriers; then the tables.
 // ---------------------------------------------------------------------------------------------
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) __nanosleep(64);
-    }
-    return false;
-}
-// CTA-wide bounded wait with a uniform result.  Only the first warp polls; the others sleep in the CTA
-// barrier instead of spinning (6 % fewer warp instructions on the 16-node workload, same run time).
-// After the barrier every other thread observes the completed phase itself with a try_wait that
-// returns at once, which makes the copies' writes visible to it.
-__device__ __forceinline__ bool cta_wait(uint32_t bar, uint32_t parity) {
-    bool ok = true;
-    if (threadIdx.x < 32) ok = mbar_wait(bar, parity);
-    ok = __syncthreads_and(ok);
-    if (ok && threadIdx.x >= 32) mbar_wait(bar, parity);
-    return ok;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-
 struct TmaGeom {
     int C;           // tile columns = boxes * box_cols
     int box_cols;    // columns per bulk copy (power of two, <= 256; 16-byte multiple)
@@ -385,7 +187,7 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < geo.stages; ++s) mbar_init(smem_u32(&bars[s]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
         for (int s = 0; s < geo.stages && s < my_tiles; ++s) issue(s, first + (long long)s * gridDim.x);
     }
     // tables staged in shared memory when small, else read from global memory (cached)
@@ -398,9 +200,10 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         if (!cta_wait(smem_u32(&bars[s]), parity)) {  // uniform decision: give up together
             if (threadIdx.x == 0) {
                 atomicExch(&g_kernel_error, 1);
-                // let copies already issued into the other stages land (bounded) before the CTA's
-                // shared memory is released
-                for (long long j = it + 1; j < my_tiles && j < it + geo.stages; ++j)
+                // Every copy this CTA has issued may still be on its way, the one that was waited for
+                // included: give each of them one more bounded wait before the CTA's shared memory is
+                // released.
+                for (long long j = it; j < my_tiles && j < it + geo.stages; ++j)
                     mbar_wait(smem_u32(&bars[j % geo.stages]), (uint32_t)((j / geo.stages) & 1));
             }
             __syncthreads();
@@ -468,238 +271,9 @@ __global__ void __launch_bounds__(kMaxThreads) step_tma_kernel(const __grid_cons
         }
         if (it + geo.stages < my_tiles) {
             // order this thread's shared-memory accesses before the bulk copy that refills the stage
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            fence_before_refill();
             __syncthreads();
             if (threadIdx.x == 0) issue(s, first + (it + geo.stages) * gridDim.x);
-        }
-    }
-}
-
-
-// ---------------------------------------------------------------------------------------------
-// Merged-staging kernel for long neighbour lists (many nodes, dense rows): ONE staged value per
-// neighbour, a branch-free weighted sum over the row, two float4 column groups per thread.
-//
-// DecentLaM.  With z_j = x_j - r (r = row 0's value of the column: a common reference that keeps z
-// small whenever the replicas are close) and v_j = g_j - z_j / gamma, Eq. (decentLaM-x-1) reads
-//     g~_i = sum_{j in N_i} w_ij v_j + z_i S_i / gamma,      S_i = sum_{j != i} w_ij + w_ii (stored),
-// (expand: sum_j w_ij g_j + (1/gamma) sum_{j != i} w_ij (z_i - z_j); the self term of the v-sum
-// cancels against w_ii z_i / gamma).  Pass 1 turns the staged (x, g) into v: in place of g for fp32
-// gradients, in a tile of its own for bf16; m is not staged, each thread reads its own m from
-// global memory while the loop runs.
-// DmSGD / DSGD.  The partial average sum_j w_ij y_j is taken as such, the self weight being the
-// exact remainder 1 - sum_{j != i} w_ij (rounded once to fp32).  Pass 1 forms y in place of x
-// (DmSGD: m' = beta m + g with m straight from global memory, y = x - gamma m'; adapt-then-combine:
-// y = x - gamma g; adapt-with-combine: y = x, no pass 1).
-// Pass 2: the L = C/8 lanes that share a row fetch its table entries together and hand them round
-// with shuffles; slots past the end of a row carry weight 0 and point at row i itself.  Tables live
-// in shared memory when they fit (the large shared-memory carve-out leaves too little L1 to keep
-// them cached otherwise).
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ float4 lds128(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(addr)
-                 : "memory");
-    return v;
-}
-
-struct MergedGeom {
-    int C;          // tile columns (power of two, 32 .. 256)
-    int cv_shift;   // log2(C / 4)
-    int tables_in_smem;
-    int prefetch_m;        // DecentLaM: request the tile's m lines into L2 before waiting for the tile
-    uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
-    uint32_t v_off, g_off; // byte offsets of the staged-value tile and of the g landing area inside the stage
-    uint32_t stage_bytes;
-    uint32_t tx_bytes;
-    long long num_tiles;
-};
-
-template <int RULE, typename GT>
-__global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant__ CUtensorMap tm_x,
-                                                           const __grid_constant__ CUtensorMap tm_g,
-                                                           dlm_step_args a, MergedGeom geo) {
-    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned char* st = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
-    uint64_t* bar_ptr = reinterpret_cast<uint64_t*>(st + geo.stage_bytes);
-    int4* s_rows = reinterpret_cast<int4*>(st + geo.stage_bytes + 16);
-    int2* s_ent = reinterpret_cast<int2*>(s_rows + a.n);
-    const uint32_t bar = smem_u32(bar_ptr);
-
-    const long long first = blockIdx.x;
-    const long long my_tiles = first < geo.num_tiles ? (geo.num_tiles - first + gridDim.x - 1) / gridDim.x : 0;
-    const int C = geo.C;
-    auto issue = [&](long long tile) {
-        const int c0 = (int)(tile * C);
-        mbar_expect_tx(bar, geo.tx_bytes);
-        tma_load_2d(smem_u32(st), &tm_x, c0, 0, bar);
-        tma_load_2d(smem_u32(st + geo.g_off), &tm_g, c0, 0, bar);
-    };
-    if (threadIdx.x == 0) {
-        mbar_init(bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (my_tiles > 0) issue(first);
-    }
-    const int4* rows = reinterpret_cast<const int4*>(a.rows);
-    const int2* ent = reinterpret_cast<const int2*>(a.ent);
-    if (geo.tables_in_smem) {  // overlaps the first copies
-        for (int r = threadIdx.x; r < a.n; r += blockDim.x) s_rows[r] = rows[r];
-        for (int p = threadIdx.x; p < a.nnz; p += blockDim.x) s_ent[p] = ent[p];
-        rows = s_rows;
-        ent = s_ent;
-    }
-    __syncthreads();
-
-    float* xs = reinterpret_cast<float*>(st);
-    float* vs = reinterpret_cast<float*>(st + geo.v_off);  // staged values: v (DecentLaM) or y (the x tile itself)
-    const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off);
-    const int items = a.n << geo.cv_shift;
-    const int cv_mask = (1 << geo.cv_shift) - 1;
-    const unsigned full = 0xffffffffu;
-    const int lshift = geo.cv_shift - 1, L = 1 << lshift;  // lanes per row in pass 2
-    const int witems = a.n << lshift, witems_padded = (witems + 31) & ~31;
-    const int lane = threadIdx.x & 31, gbase = lane & ~(L - 1), glane = lane & (L - 1);
-    const uint32_t row_bytes = (uint32_t)C * 4;
-
-    constexpr int kPre = 4;  // pass-1 items per thread whose m is fetched ahead (all of them at 512 threads)
-    for (long long it = 0; it < my_tiles; ++it) {
-        const long long tile_base = (first + it * gridDim.x) * C;
-        // DmSGD reads m in pass 1, straight from global memory: issue those loads before waiting for
-        // the tile, so that their latency hides behind the copies instead of stalling every item
-        Pack<4> mpre[kPre];
-        if (RULE == DLM_RULE_DMSGD) {
-#pragma unroll
-            for (int k = 0; k < kPre; ++k) {
-                const int e = threadIdx.x + k * blockDim.x;
-                const long long c = tile_base + (e & cv_mask) * 4;
-                mpre[k] = {{0.f, 0.f, 0.f, 0.f}};
-                if (e < items && c < a.d) mpre[k] = ld_f32<4>(a.m + (size_t)(e >> geo.cv_shift) * a.ld + c);
-            }
-        }
-        if (LAM && geo.prefetch_m) {
-            // DecentLaM reads m in pass 2, one load per item just before its mixing loop, too short a loop
-            // to cover a trip to DRAM.  Ask for those lines now, while the tile is still on its way: the
-            // prefetch holds no registers and the later load finds its line in L2.  One request for each
-            // end of every 128-byte row segment (a segment may straddle two lines).
-            const int seg_shift = geo.cv_shift - 3, segs = a.n << seg_shift;  // C / 32 segments per row
-            for (int e = threadIdx.x; e < 2 * segs; e += blockDim.x) {
-                const int sg = e >> 1;
-                const long long c = tile_base + (long long)(sg & ((1 << seg_shift) - 1)) * 32 + (e & 1) * 28;
-                if (c < a.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.m + (size_t)(sg >> seg_shift) * a.ld + c));
-            }
-        }
-        if (!cta_wait(bar, (uint32_t)(it & 1))) {  // uniform decision: give up together
-            if (threadIdx.x == 0) atomicExch(&g_kernel_error, 3);
-            return;                          // single stage: no other copy of this CTA is in flight
-        }
-        if (RULE != DLM_RULE_DSGD_AWC) {  // pass 1 (the adapt-with-combine rule averages x as it is)
-            int k = 0;
-            for (int e = threadIdx.x; e < items; e += blockDim.x, ++k) {
-                const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
-                const Pack<4> xi = ld_f32<4>(xs + i * C + off);
-                const Pack<4> gi = ld_g<4>(gs + i * C + off);
-                Pack<4> v;
-                if (LAM) {  // v = g - (x - r) / gamma
-                    const Pack<4> ref = ld_f32<4>(xs + off);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
-                } else if (RULE == DLM_RULE_DMSGD) {  // m' = beta m + g ; y = x - gamma m'
-                    const long long c = tile_base + off;
-                    Pack<4> mi = {{0.f, 0.f, 0.f, 0.f}}, mn;
-                    if (k < kPre) {
-                        mi = k == 0 ? mpre[0] : k == 1 ? mpre[1] : k == 2 ? mpre[2] : mpre[3];
-                    } else if (c < a.d) {
-                        mi = ld_f32<4>(a.m + (size_t)i * a.ld + c);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], v.v[u]);
-                    if (c < a.d) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
-                } else {  // adapt-then-combine: y = x - gamma g
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.gamma, gi.v[u], xi.v[u]);
-                }
-                st_f32<4>(vs + i * C + off, v);
-            }
-            __syncthreads();
-        }
-        // pass 2
-        for (int e = threadIdx.x; e < witems_padded; e += blockDim.x) {
-            const bool live = e < witems;
-            const int slot = live ? (e >> lshift) : 0;
-            const int4 ri = rows[slot];
-            const int i = ri.x, len = ri.z;
-            // column groups {q, q + L}; with four lanes per row, neighbouring rows take the two
-            // halves in opposite order so that a quarter warp still covers all 32 banks
-            const int par = (L == 4) ? (slot & 1) : 0;
-            const int off0 = (L == 4 ? glane + 4 * par : glane) * 4;
-            const int off1 = (L == 4 ? glane + 4 * (1 - par) : glane + L) * 4;
-            const long long c0 = tile_base + off0, c1 = tile_base + off1;
-            const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;
-            Pack<4> m0 = {{0.f, 0.f, 0.f, 0.f}}, m1 = {{0.f, 0.f, 0.f, 0.f}};
-            if (LAM) {
-                if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
-                if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
-            }
-            // the averaging rules replace the stored diagonal by the exact remainder 1 - sum_{j != i} w_ij
-            const int self_bits = LAM ? 0 : a.selfw[slot];
-            float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-            const uint32_t vb0 = smem_u32(vs) + off0 * 4, vb1 = smem_u32(vs) + off1 * 4;
-            const int len_max = __reduce_max_sync(full, len);
-            for (int base0 = 0; base0 < len_max; base0 += L) {
-                int2 en = make_int2(i, 0);  // filler: adds exactly 0 * (staged value of row i)
-                if (base0 + glane < len) {
-                    en = ent[ri.y + base0 + glane];
-                    if (!LAM && en.x == i) en.y = self_bits;
-                }
-                // DecentLaM keeps whole groups of four (no remainder loop: its m loads are in flight and
-                // registers are short); the averaging rules stop at the longest row of the warp
-                const int cnt = LAM ? min(L, (len_max - base0 + 3) & ~3) : min(L, len_max - base0);
-#pragma unroll 4
-                for (int r = 0; r < cnt; ++r) {
-                    const int j = __shfl_sync(full, en.x, gbase + r);
-                    const float w = __int_as_float(__shfl_sync(full, en.y, gbase + r));
-                    const float4 v0 = lds128(vb0 + (uint32_t)j * row_bytes);
-                    const float4 v1 = lds128(vb1 + (uint32_t)j * row_bytes);
-                    acc0[0] = fmaf(w, v0.x, acc0[0]); acc0[1] = fmaf(w, v0.y, acc0[1]);
-                    acc0[2] = fmaf(w, v0.z, acc0[2]); acc0[3] = fmaf(w, v0.w, acc0[3]);
-                    acc1[0] = fmaf(w, v1.x, acc1[0]); acc1[1] = fmaf(w, v1.y, acc1[1]);
-                    acc1[2] = fmaf(w, v1.z, acc1[2]); acc1[3] = fmaf(w, v1.w, acc1[3]);
-                }
-            }
-            const float S_i = __int_as_float(ri.w);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int off = h ? off1 : off0;
-                Pack<4> xn;
-                if (LAM) {
-                    const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
-                    Pack<4> mn;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, h ? acc1[u] : acc0[u]);
-                        mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
-                        xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
-                    }
-                    if (h ? st1 : st0) st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
-                } else {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) xn.v[u] = h ? acc1[u] : acc0[u];
-                    if (RULE == DLM_RULE_DSGD_AWC) {
-                        const Pack<4> gi = ld_g<4>(gs + i * C + off);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
-                    }
-                }
-                if (h ? st1 : st0) st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
-            }
-        }
-        if (it + 1 < my_tiles) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncthreads();
-            if (threadIdx.x == 0) issue(first + (it + 1) * gridDim.x);
         }
     }
 }
@@ -707,80 +281,7 @@ __global__ void __launch_bounds__(512) step_merged_kernel(const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-struct DeviceInfo {
-    int sms = 0;
-    int smem_optin = 0;
-    bool ok = false;
-};
-
-const DeviceInfo& device_info() {
-    static DeviceInfo info[64];
-    static std::mutex mu;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
-        static DeviceInfo bad;
-        return bad;
-    }
-    std::lock_guard<std::mutex> lock(mu);
-    if (!info[dev].ok) {
-        cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&info[dev].smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        info[dev].ok = info[dev].sms > 0;
-    }
-    return info[dev];
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            cudaGetLastError();
-    });
-    return fn;
-}
-
-// 2-D map over a row-major [n, d] array with row stride ld elements; box = [n rows (or box_rows), C columns].
-bool make_map(CUtensorMap* map, const void* ptr, bool bf16, int n, int64_t d, int64_t ld, int C, int box_rows = 0) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t esz = bf16 ? 2 : 4;
-    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
-    cuuint32_t box[2] = {(cuuint32_t)C, (cuuint32_t)(box_rows > 0 ? box_rows : n)};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-                    const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
-int ilog2(int v) {
-    int l = 0;
-    while ((1 << (l + 1)) <= v) ++l;
-    return l;
-}
-
 size_t table_bytes(const dlm_step_args& a) { return (size_t)(2 * a.n + 1) * 4 + (size_t)a.nnz * 8; }
-
-int g_tune_path = 0;    // 0 auto, 1 force tile kernel, 2 force pipeline kernel (error if ineligible)
-int g_tune_cols = 0;    // tile columns, 0 = auto
-int g_tune_stages = 0;  // pipeline stages, 0 = auto
-int g_tune_ctas = 0;    // CTAs per SM, 0 = auto
-int g_tune_threads = 0;  // pipeline kernel block size (128, 256 or 512), 0 = auto
-int g_tune_mix = 0;     // 0 auto, 1 pipeline kernel with the plain mixing loop, 2 merged-staging kernel
-int g_tune_tables = 0;  // 0 auto, 1 stage tables in shared memory, 2 read them from global memory
-int g_tune_tiles_per_cta = 0;  // 0 = auto; t > 0: ceil(tiles / t) CTAs; t < 0: persistent grid of sms * ctas
 
 template <int RULE, typename GT, int VEC>
 int launch_tile(const dlm_step_args& a, cudaStream_t stream) {
@@ -924,62 +425,6 @@ int launch_tma_plain(const dlm_step_args& a, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
 
-// Merged staging (long rows).  DLM_ERR_UNSUPPORTED if the shape does not fit.
-template <int RULE, typename GT>
-int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
-    const DeviceInfo& dev = device_info();
-    if (!dev.ok) return DLM_ERR_CUDA;
-    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
-    const bool bf16 = sizeof(GT) == 2;
-    if (a.n > 256 || a.d > 0x7fffffffLL - 4096) return DLM_ERR_UNSUPPORTED;
-    int C = 1 << ilog2(std::max(1, (int)(32768 / ((size_t)a.n * 4))));
-    C = std::max(32, std::min(256, C));
-    if (g_tune_cols >= 32 && g_tune_cols <= 256 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
-    const size_t tab = (size_t)a.n * 16 + (size_t)a.nnz * 8;
-    MergedGeom geo;
-    size_t smem = 0;
-    for (;; C /= 2) {
-        if (C < 32) return DLM_ERR_UNSUPPORTED;
-        const size_t xb = ((size_t)a.n * C * 4 + 127) & ~(size_t)127;
-        const size_t gb = ((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127;
-        geo.x_bytes = (uint32_t)xb;
-        if (LAM) {  // [x | v | g]: for fp32 gradients v overwrites g in place
-            geo.v_off = (uint32_t)xb;
-            geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);
-            geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
-        } else {    // [x (becomes y) | g]
-            geo.v_off = 0;
-            geo.g_off = (uint32_t)xb;
-            geo.stage_bytes = (uint32_t)(xb + gb);
-        }
-        // tables in shared memory if two CTAs per SM still fit, or on request
-        const size_t fixed = 128 + 16 + 16;
-        const size_t with_tab = fixed + geo.stage_bytes + tab;
-        geo.tables_in_smem = g_tune_tables == 2 ? 0 : (with_tab <= (size_t)dev.smem_optin / 2 - 1024 || g_tune_tables == 1);
-        smem = geo.tables_in_smem ? with_tab : fixed + geo.stage_bytes;
-        if (smem <= (size_t)dev.smem_optin / 2 - 1024 || (C == 32 && smem <= (size_t)dev.smem_optin)) break;
-    }
-    geo.C = C;
-    geo.cv_shift = ilog2(C / 4);
-    // measured: +3 to +8 % with tiles of 64 columns or more (up to 128 nodes); with 256 nodes and
-    // 32-column tiles the extra requests cost 6 % instead
-    geo.prefetch_m = C >= 64;
-    geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
-    geo.num_tiles = (a.d + C - 1) / C;
-    CUtensorMap tm_x, tm_g;
-    if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, C) || !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, C))
-        return DLM_ERR_UNSUPPORTED;
-    auto kern = step_merged_kernel<RULE, GT>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return DLM_ERR_CUDA;
-    const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : (geo.tables_in_smem ? 8 : 4);
-    const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
-    const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512) ? g_tune_threads : 512;
-    kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_g, a, geo);
-    dlm_count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
-}
-
 // Long rows take the merged-staging kernel when the shape allows it, everything else the pipeline
 // kernel with the plain mixing loop.
 template <int RULE, typename GT>
@@ -993,9 +438,9 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     // one staged array and no momentum in pass 2: up to 128 nodes DmSGD and adapt-then-combine DSGD gain
     // 1 to 7 % from six entries per row on (exponential graphs of 32 and 64 nodes)
     if ((RULE == DLM_RULE_DMSGD || RULE == DLM_RULE_DSGD_ATC) && a.n <= 128 && a.max_degree >= 6) want_merged = true;
-    const bool merged = g_tune_mix == 2 ? true : g_tune_mix == 1 ? false : want_merged;
+    const bool merged = (g_tune_mix == 2 || g_tune_mix == 3) ? true : g_tune_mix == 1 ? false : want_merged;
     if (merged) {
-        int rc = launch_merged<RULE, GT>(a, stream);
+        int rc = dlm_launch_merged(RULE, a, stream);
         if (rc != DLM_ERR_UNSUPPORTED) return rc;
     }
     // DmSGD on 257 .. 511 nodes: the plain-load kernel stages one array where the bulk-copy kernel stages
@@ -1080,14 +525,16 @@ int dlm_step_set_tuning(int knob, int value) {
     }
 }
 
-// Reads and clears the error flag of the step kernels' bounded waits.
+// Reads and clears the error flags of the step kernels' bounded waits (this file's and the merged kernel's).
 int dlm_step_take_error(int* flag) {
-    int v = 0;
+    int v = 0, merged = 0;
     if (cudaMemcpyFromSymbol(&v, g_kernel_error, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
     if (v != 0) {
         int zero = 0;
         if (cudaMemcpyToSymbol(g_kernel_error, &zero, sizeof(int)) != cudaSuccess) return DLM_ERR_CUDA;
     }
-    *flag = v;
+    int rc = dlm_merged_take_error(&merged);
+    if (rc != DLM_OK) return rc;
+    *flag = v != 0 ? v : merged;
     return DLM_OK;
 }

@@ -59,6 +59,56 @@ std::vector<Edge> unique_neighbours(int i, const std::vector<int32_t>& js, int q
     return nb;
 }
 
+// Compact tables of the merged DecentLaM kernel: 4 bytes per row, 2 bytes per off-diagonal entry
+// {column, index into the table of distinct weights}.  Built when they can represent the slot exactly:
+// at most 256 nodes, 255 distinct off-diagonal weights (bit patterns), 65535 off-diagonal entries,
+// rows of at most 255 neighbours.
+void make_compact(dlm_slot& s) {
+    const int n = (int)s.rowptr.size() - 1;
+    s.compact.clear();
+    s.compact_nw = s.compact_noff = 0;
+    if (n > 256) return;
+    std::vector<uint32_t> lut;  // distinct off-diagonal weight bit patterns, in order of first use
+    std::vector<uint16_t> cent;
+    std::vector<uint32_t> rowrec(n);
+    std::vector<float> S(n), wself(n);
+    for (int r = 0; r < n; ++r) {
+        const int i = s.order[r];
+        const size_t first = cent.size();
+        float diag = 0.0f;
+        for (int32_t p = s.rowptr[i]; p < s.rowptr[i + 1]; ++p) {
+            if (s.col[p] == i) {
+                diag = s.val[p];
+                continue;
+            }
+            uint32_t bits;
+            std::memcpy(&bits, &s.val[p], sizeof(bits));
+            size_t w = std::find(lut.begin(), lut.end(), bits) - lut.begin();
+            if (w == lut.size()) {
+                if (lut.size() == 255) return;
+                lut.push_back(bits);
+            }
+            cent.push_back((uint16_t)(s.col[p] | (w << 8)));
+        }
+        const size_t len = cent.size() - first;
+        if (len > 255 || first > 65535 || cent.size() > 65535) return;
+        rowrec[r] = (uint32_t)i | ((uint32_t)len << 8) | ((uint32_t)first << 16);
+        std::memcpy(&S[r], &s.rows[4 * r + 3], sizeof(float));
+        wself[r] = diag;
+    }
+    const size_t nw = lut.size();
+    const size_t bytes = (size_t)12 * n + 4 * (nw + 1) + 2 * cent.size();
+    s.compact.assign((bytes + 15) & ~(size_t)15, 0);
+    unsigned char* b = s.compact.data();
+    std::memcpy(b, rowrec.data(), 4 * (size_t)n);
+    std::memcpy(b + 4 * (size_t)n, S.data(), 4 * (size_t)n);
+    std::memcpy(b + 8 * (size_t)n, wself.data(), 4 * (size_t)n);
+    if (nw) std::memcpy(b + 12 * (size_t)n, lut.data(), 4 * nw);  // entry nw stays 0.0f: the filler's weight
+    if (!cent.empty()) std::memcpy(b + 12 * (size_t)n + 4 * (nw + 1), cent.data(), 2 * cent.size());
+    s.compact_nw = (int)nw;
+    s.compact_noff = (int)cent.size();
+}
+
 // Processing order for the kernels: rows of similar length next to each other, so that the rows
 // sharing a warp run the same number of neighbour iterations.
 void make_order(dlm_slot& s) {
@@ -90,6 +140,7 @@ void make_order(dlm_slot& s) {
         s.ent[2 * p] = s.col[p];
         std::memcpy(&s.ent[2 * p + 1], &s.val[p], sizeof(float));
     }
+    make_compact(s);
 }
 
 int upload(dlm_slot& s) {
@@ -101,6 +152,11 @@ int upload(dlm_slot& s) {
         return DLM_ERR_CUDA;
     if (cudaMemcpy(s.d_ent, s.ent.data(), s.ent.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return DLM_ERR_CUDA;
+    if (!s.compact.empty()) {
+        if (cudaMalloc((void**)&s.d_compact, s.compact.size()) != cudaSuccess) return DLM_ERR_CUDA;
+        if (cudaMemcpy(s.d_compact, s.compact.data(), s.compact.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+            return DLM_ERR_CUDA;
+    }
     if (cudaMalloc((void**)&s.d_selfw, s.selfw.size() * sizeof(int32_t)) != cudaSuccess) return DLM_ERR_CUDA;
     if (cudaMemcpy(s.d_selfw, s.selfw.data(), s.selfw.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return DLM_ERR_CUDA;
@@ -366,6 +422,7 @@ int topology_destroy(dlm_topology* topo) {
         if (s.d_rows) cudaFree(s.d_rows);
         if (s.d_ent) cudaFree(s.d_ent);
         if (s.d_selfw) cudaFree(s.d_selfw);
+        if (s.d_compact) cudaFree(s.d_compact);
         if (s.d_rowptr) cudaFree(s.d_rowptr);
         if (s.d_col) cudaFree(s.d_col);
         if (s.d_val) cudaFree(s.d_val);

@@ -45,9 +45,32 @@ def rel_l2(a, o):
 
 
 def to64(t):
-    """torch tensor (fp32 or bf16, any device) -> float64 numpy (exact)."""
+    """torch tensor (fp32 or bf16, any device) -> float64 numpy (exact).  bf16 values are handed over as
+    their bit patterns and widened by the oracle's own helper, so no conversion of torch's takes part."""
     import torch
+    if t.dtype == torch.bfloat16:
+        bits = t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+        return oracle.bf16_to_f64(bits).reshape(tuple(t.shape))
     return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def bf16_tensor(g32, device):
+    """The harness's rounding of fp32 gradients to bfloat16: round to nearest, ties to even, done by
+    inputs.f32_to_bf16_bits on the host (pinned bit by bit in test_bf16_rounding.py); returns a torch
+    bfloat16 tensor on `device` holding exactly those bits."""
+    import torch
+    bits = inputs.f32_to_bf16_bits(np.asarray(g32, dtype=np.float32))
+    return torch.from_numpy(bits.view(np.int16).copy()).to(device).view(torch.bfloat16)
+
+
+def assert_device_rounding_is_rne(g32_t, gb_t, n_check=1 << 16):
+    """Where a full-size gradient is rounded to bfloat16 on the device (torch's conversion), check on a
+    strided sample that it produced the bits inputs.f32_to_bf16_bits gives for the same fp32 values."""
+    flat32, flatb = g32_t.reshape(-1), gb_t.reshape(-1)
+    step = max(1, flat32.numel() // n_check)
+    want = inputs.f32_to_bf16_bits(flat32[::step].cpu().numpy())
+    got = flatb[::step].contiguous().view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(want, got)
 
 
 def oracle_rule(rule, W, x, m, g, beta, gamma, threads=THREADS):

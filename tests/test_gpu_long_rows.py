@@ -28,6 +28,24 @@ SHAPES = [("er_mh", 64, 0.15, 1_500_008), ("er_mh", 128, 0.10, 600_008), ("stati
 @pytest.mark.parametrize("rule", ["decentlam", "dmsgd", "dsgd_atc"])
 @pytest.mark.parametrize("topology,n,er_p,d", SHAPES)
 def test_long_rows_sampled(topology, n, er_p, d, rule, g_dtype):
+    _run(topology, n, er_p, d, rule, g_dtype)
+
+
+@pytest.mark.parametrize("threads", [256, 384, 512])
+@pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("topology,n,er_p,d", SHAPES + [("er_mh", 256, 0.05, 300_008), ("ring", 200, 0.0, 200_008)])
+def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, threads):
+    """The compact-table form of the merged DecentLaM kernel (2-byte entries, per-lane entry loads, self term
+    added last), forced by knob 7 = 3 at each of its block sizes."""
+    from paper_2104_11981_b200 import binding as B
+    try:
+        B.set_tuning(7, 3); B.set_tuning(12, threads)
+        _run(topology, n, er_p, d, "decentlam", g_dtype)
+    finally:
+        B.set_tuning(7, 0); B.set_tuning(12, 0)
+
+
+def _run(topology, n, er_p, d, rule, g_dtype):
     from paper_2104_11981_b200 import binding as B
     dev = torch.device("cuda:0")
     steps = 12

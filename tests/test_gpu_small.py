@@ -6,15 +6,11 @@ import pytest
 import torch
 
 import oracle
-from helpers import build_both, lib_rule, oracle_rule, rel_l2, to64
+from helpers import bf16_tensor, build_both, lib_rule, oracle_rule, rel_l2, to64
 from paper_2104_11981_b200 import inputs
 
 pytestmark = pytest.mark.gpu
-TOL_STEP = 1e-6      # relative L2 per step, x and m
-# A tensor of a handful of elements does not average rounding errors: one fp32 cancellation of
-# x against gamma*m' (or of the consensus differences) costs |operand| / |result| ulps on that
-# element.  Below 4096 elements the bound is therefore loosened to 5e-6.
-TOL_STEP_TINY = 5e-6
+TOL_STEP = 1e-6      # relative L2 per step against the oracle, x and m (the stated tolerance)
 GUARD = 64
 CANARY = 1234.5
 
@@ -33,6 +29,22 @@ def _canaries_intact(flat, n, d, ld, offset):
     return ok and bool((body[:, d:] == CANARY).all())
 
 
+def _widened(rule, topology, n, d, k, consensus):
+    """The few cases whose error is judged against the larger of the result and the operand it was formed
+    from, as (reason, tolerance); None = the plain relative L2 against the oracle at 1e-6 applies (every
+    other case of this file measured 7e-7 or less that way)."""
+    if topology == "complete" and n * d < 16:
+        return ("two elements: x' = x - gamma m' cancels half of x on both at once, and a tensor this small "
+                "has no other elements to average the one rounding error over", 5e-6)
+    if topology == "complete" and n >= 256 and k == 0:
+        return ("complete graph of 256+ nodes fed independent random rows: the step contracts x onto its mean, "
+                "so the result is ~1/sqrt(n) of the operands whose fp32 roundings it inherits", 1e-6)
+    if topology == "er_mh" and n >= 256 and consensus and k == 1:
+        return ("dense graph one step after a consensus start with random momenta: m' = beta m + g~ cancels "
+                "most of m (the method's consensus correction), the result is ~1/4 of the operands", 1e-6)
+    return None
+
+
 def _case(rule, topology, n, d, g_dtype, ld=None, offset=0, seed=0, steps=3, beta=0.9, gamma=0.1, consensus=False):
     from paper_2104_11981_b200 import binding as B
     dev = torch.device("cuda:0")
@@ -47,20 +59,22 @@ def _case(rule, topology, n, d, g_dtype, ld=None, offset=0, seed=0, steps=3, bet
     worst = 0.0
     for k in range(steps):
         g32 = inputs.normal_np((n, d), 1e-3, seed + 10 + k)
-        g, gf = _padded(n, d, ld, offset, dev, torch.from_numpy(g32).to(dev).to(gt), gt)
+        g_fill = bf16_tensor(g32, dev) if g_dtype == "bf16" else torch.from_numpy(g32).to(dev)
+        g, gf = _padded(n, d, ld, offset, dev, g_fill, gt)
         x_in, m_in = to64(x), to64(m)
         xo, mo = oracle_rule(rule, Ws[k % len(Ws)], x_in, m_in, to64(g), np.float32(beta), np.float32(gamma))
         g_before = g.clone()
         lib_rule(rule, topo, k, x, m, g, beta, gamma)
         torch.cuda.synchronize()
         assert B.kernel_error() == 0
-        # errors are measured against the larger of the result and the state it was formed from:
-        # on dense graphs m' = beta m + g~ cancels most of a random m (that is the method's
-        # consensus correction), which would otherwise inflate a purely relative figure
-        ex = np.linalg.norm(to64(x) - xo) / max(np.linalg.norm(xo), np.linalg.norm(x_in), 1e-300)
-        em = np.linalg.norm(to64(m) - mo) / max(np.linalg.norm(mo), float(beta) * np.linalg.norm(m_in), 1e-300)
+        wide = _widened(rule, topology, n, d, k, consensus)
+        if wide is None:
+            ex, em, tol = rel_l2(to64(x), xo), rel_l2(to64(m), mo), TOL_STEP
+        else:
+            ex = np.linalg.norm(to64(x) - xo) / max(np.linalg.norm(xo), np.linalg.norm(x_in), 1e-300)
+            em = np.linalg.norm(to64(m) - mo) / max(np.linalg.norm(mo), float(beta) * np.linalg.norm(m_in), 1e-300)
+            tol = wide[1]
         worst = max(worst, ex, em)
-        tol = TOL_STEP if n * d >= 4096 else TOL_STEP_TINY
         assert ex <= tol and em <= tol, (rule, topology, n, d, g_dtype, k, ex, em)
         assert torch.equal(g, g_before)
         assert _canaries_intact(xf, n, d, ld, offset) and _canaries_intact(mf, n, d, ld, offset)
@@ -233,6 +247,18 @@ def test_bf16_path_equals_f32_path_on_prerounded_gradients():
         lib_rule(rule, topo, 0, xb, mb, gf, 0.9, 0.05)
         torch.cuda.synchronize()
         assert torch.equal(xa, xb) and torch.equal(ma, mb)
+
+
+def test_device_bf16_conversion_is_the_harness_rounding():
+    """Large gradients are rounded to bfloat16 on the device by torch's conversion; it must give the bit
+    patterns of the harness's pinned host rounding (nearest, ties to even), planted ties included."""
+    dev = torch.device("cuda:0")
+    bits = inputs.normal_np((1 << 20,), 1e-3, 51).view(np.uint32).copy()
+    bits[: 1 << 12] = (bits[: 1 << 12] & np.uint32(0xFFFF0000)) | np.uint32(0x8000)      # exact ties, both parities
+    f = bits.view(np.float32)
+    got = torch.from_numpy(f).to(dev).to(torch.bfloat16).view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, inputs.f32_to_bf16_bits(f))
+    assert np.array_equal(to64(bf16_tensor(f, dev)), oracle.bf16_to_f64(inputs.f32_to_bf16_bits(f)))
 
 
 def test_hand_example_on_gpu():
