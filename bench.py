@@ -43,6 +43,9 @@ def parse_args():
                     help="node-sharded run over this many ranks (the paper's deployment): under torchrun with --gpus N "
                          "ranks exchange halo rows over NCCL; on one GPU rank 0's share is timed with device copies "
                          "standing in for the link")
+    ap.add_argument("--tuning", default="",
+                    help="expert launch-shape knobs of dlm_set_tuning as 'knob=value,...' (results do not depend on them "
+                         "beyond rounding); for profiler captures and sweeps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the DmSGD / PmSGD side timings")
@@ -385,6 +388,9 @@ def run_ours(args):
     gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
 
     topo = build_topology(B, inputs, args.workload)
+    for item in filter(None, args.tuning.split(",")):
+        knob, value = item.split("=")
+        B.set_tuning(int(knob), int(value))
 
     x0 = inputs.normal_torch((n, d), w.x0_std, inputs.seed_for(args.workload, inputs.P_X0) + rank, dev)
     x = torch.empty_like(x0); m = torch.empty_like(x0)
@@ -508,7 +514,8 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else ""), "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
+            "config": {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else "") +
+                                   (f" (tuning {args.tuning})" if args.tuning else ""), "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
                        "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

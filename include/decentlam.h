@@ -403,17 +403,19 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 5  neighbour tables: 1 = staged in shared memory, 2 = read from global memory
  *   knob 6  threads per CTA of the pipeline kernels (128, 256 or 512)
  *   knob 7  1 = pipeline kernel with the plain mixing loop, 2 = merged-staging kernel (one staged
- *           value per neighbour), 3 = its compact-table form for decentlam_step where the graph allows it
+ *           value per neighbour) with 8-byte table entries, 3 = merged-staging kernel, for decentlam_step
+ *           in its compact-table form where the graph allows it (the automatic choice on long rows)
  *   knob 8  lsq_grad and lsq_grad_gram: row chunks per node (at most 64)
  *   knob 9  lsq_grad: 2 = register-pipelined kernel instead of the bulk-copy pipeline
  *   knob 10 pmsgd_step: blocks per SM of a capped grid (default: one thread per 4 columns, uncapped)
  *   knob 11 lsq_grad_gram: share of H kept in L2 with evict-last priority between calls, in 1/1000
  *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
  *           size, else none)
- *   knob 12 block size of the compact-table merged kernel (256, 384 or 512)
- * Results do not depend on the knobs, with one exception: the merged-staging kernel (knob 7 = 2,
- * the default on long rows: 12 or more entries, 8 or more for dmsgd_step and up to 128 nodes) arranges the same sum differently and
- * agrees with the other paths to rounding, not bitwise.  DLM_ERR_KIND for an unknown knob.
+ *   knob 12 block size of the compact-table merged kernel (128, 256, 384 or 512)
+ * Results do not depend on the knobs, with one exception: the merged-staging kernels (knob 7 = 2 or 3,
+ * the default on long rows: 8 or more entries; 12 or more for dsgd_step above 128 nodes) arrange the same
+ * sum differently and agree with the other paths, and with each other, to rounding, not bitwise.
+ * DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);
 

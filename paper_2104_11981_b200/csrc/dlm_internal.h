@@ -124,6 +124,6 @@ int dlm_launch_shard_step(int rule, const dlm_shard_args& a, void* stream);  // 
 int dlm_launch_local_momentum(int rows, int64_t d, int64_t ld, float* x, float* m, const void* g, int g_dtype,
                               int64_t ldg, float beta, float gamma, void* stream);
 int dlm_shard_take_error(int* flag);
-int dlm_compact_set_threads(int value);
+int dlm_compact_set_tuning(int knob, int value);
 
 void dlm_count_launch(int launches);

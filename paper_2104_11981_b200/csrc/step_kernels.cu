@@ -434,6 +434,10 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     // single array either way and gains from the merged pass already at 8 entries per row.
     bool want_merged = a.max_degree >= 12 || (a.max_degree >= 8 && a.n <= 128);
     if (a.n > 128 && (long long)a.nnz < 8LL * a.n) want_merged = false;
+    // DecentLaM with compact tables (2-byte entries, three CTAs per SM at 256 nodes): ahead of the plain loop
+    // from 8 entries per row on at every size measured (static exponential graph of 256 nodes +10 %,
+    // Erdos-Renyi graphs +25 to +40 %), level with it at 7 (exponential graph of 64 nodes), behind at 3 .. 6
+    if (RULE == DLM_RULE_DECENTLAM && a.compact) want_merged = a.max_degree >= 8;
     if (RULE == DLM_RULE_DMSGD) want_merged = a.max_degree >= 8;
     // one staged array and no momentum in pass 2: up to 128 nodes DmSGD and adapt-then-combine DSGD gain
     // 1 to 7 % from six entries per row on (exponential graphs of 32 and 64 nodes)

@@ -29,11 +29,14 @@ using namespace dlm;
 __device__ int g_shard_kernel_error = 0;  // set to a non-zero code if a bounded wait ran out
 
 struct HaloGeom {
-    int C;         // tile columns (power of two, 32 .. 256)
-    int cv_shift;  // log2(C / 4)
+    int C;         // tile columns = boxes * box_cols
+    int box_cols;  // columns per bulk copy (power of two, 32 .. 256); each copy lands as a dense [rows][box_cols] sub-tile
+    int boxes;
+    int cv_shift;  // log2(box_cols / 4)
     int tables_in_smem;
-    uint32_t g_off, m_off;  // byte offsets of the g and m tiles inside the stage (128-byte multiples)
-    uint32_t halo_x_off, halo_g_off;  // byte offsets of the halo rows inside the x and g tiles
+    uint32_t sub_x, sub_g, sub_m;     // bytes per sub-tile of x (own + halo rows), g (same rows), m (own rows): 128-byte multiples
+    uint32_t g_off, m_off;            // byte offsets of the first g and m sub-tiles inside the stage
+    uint32_t halo_x_off, halo_g_off;  // byte offsets of the halo rows inside an x and a g sub-tile
     uint32_t stage_bytes;
     uint32_t tx_bytes;
     long long num_tiles;
@@ -69,16 +72,18 @@ __global__ void __launch_bounds__(512) step_halo_kernel(const __grid_constant__ 
 
     const long long first = blockIdx.x;
     const long long my_tiles = first < geo.num_tiles ? (geo.num_tiles - first + gridDim.x - 1) / gridDim.x : 0;
-    const int C = geo.C;
+    const int C = geo.C, Cb = geo.box_cols;
     auto issue = [&](long long tile) {
-        const int c0 = (int)(tile * C);
         mbar_expect_tx(bar, geo.tx_bytes);
-        tma_load_2d(smem_u32(st), &tm_x, c0, 0, bar);
-        if (halo > 0) tma_load_2d(smem_u32(st + geo.halo_x_off), &tm_hx, c0, 0, bar);
-        if (LAM) {
-            tma_load_2d(smem_u32(st + geo.g_off), &tm_g, c0, 0, bar);
-            if (halo > 0) tma_load_2d(smem_u32(st + geo.g_off + geo.halo_g_off), &tm_hg, c0, 0, bar);
-            tma_load_2d(smem_u32(st + geo.m_off), &tm_m, c0, 0, bar);
+        for (int b = 0; b < geo.boxes; ++b) {
+            const int c0 = (int)(tile * C) + b * Cb;
+            tma_load_2d(smem_u32(st + b * geo.sub_x), &tm_x, c0, 0, bar);
+            if (halo > 0) tma_load_2d(smem_u32(st + b * geo.sub_x + geo.halo_x_off), &tm_hx, c0, 0, bar);
+            if (LAM) {
+                tma_load_2d(smem_u32(st + geo.g_off + b * geo.sub_g), &tm_g, c0, 0, bar);
+                if (halo > 0) tma_load_2d(smem_u32(st + geo.g_off + b * geo.sub_g + geo.halo_g_off), &tm_hg, c0, 0, bar);
+                tma_load_2d(smem_u32(st + geo.m_off + b * geo.sub_m), &tm_m, c0, 0, bar);
+            }
         }
     };
     if (threadIdx.x == 0) {
@@ -89,10 +94,7 @@ __global__ void __launch_bounds__(512) step_halo_kernel(const __grid_constant__ 
     const auto t = stage_tables<LAM>(a, tab, geo.tables_in_smem != 0);  // overlaps the first copies
     __syncthreads();
 
-    const float* xs = reinterpret_cast<const float*>(st);
-    const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off);
-    const float* ms = reinterpret_cast<const float*>(st + geo.m_off);
-    const int items = a.n << geo.cv_shift;
+    const int items = a.n << geo.cv_shift;  // per sub-tile
     const int cv_mask = (1 << geo.cv_shift) - 1;
 
     for (long long it = 0; it < my_tiles; ++it) {
@@ -107,20 +109,26 @@ __global__ void __launch_bounds__(512) step_halo_kernel(const __grid_constant__ 
             __syncthreads();
             return;
         }
-        for (int e = threadIdx.x; e < items; e += blockDim.x) {
-            const int i = t.order[e >> geo.cv_shift], off = (e & cv_mask) * 4;
-            const long long c = tile_base + off;
-            if (c < a.d) {  // columns past d hold the copies' zero fill
-                Pack<4> xn;
-                if constexpr (LAM) {
-                    const Pack<4> mi = ld_f32<4>(ms + i * C + off);
-                    Pack<4> mn;
-                    decentlam_item<4, GT>(t, i, off, C, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
-                    store_group(a.m + (size_t)i * a.ld, c, a.d, mn);
-                } else {
-                    dmsgd_item<4>(t, i, off, C, xs, xn);
+        for (int b = 0; b < geo.boxes; ++b) {
+            const float* xs = reinterpret_cast<const float*>(st + b * geo.sub_x);
+            const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off + b * geo.sub_g);
+            const float* ms = reinterpret_cast<const float*>(st + geo.m_off + b * geo.sub_m);
+            const long long c_base = tile_base + (long long)b * Cb;
+            for (int e = threadIdx.x; e < items; e += blockDim.x) {
+                const int i = t.order[e >> geo.cv_shift], off = (e & cv_mask) * 4;
+                const long long c = c_base + off;
+                if (c < a.d) {  // columns past d hold the copies' zero fill
+                    Pack<4> xn;
+                    if constexpr (LAM) {
+                        const Pack<4> mi = ld_f32<4>(ms + i * Cb + off);
+                        Pack<4> mn;
+                        decentlam_item<4, GT>(t, i, off, Cb, xs, gs, mi, a.beta, a.gamma, a.inv_gamma, mn, xn);
+                        store_group(a.m + (size_t)i * a.ld, c, a.d, mn);
+                    } else {
+                        dmsgd_item<4>(t, i, off, Cb, xs, xn);
+                    }
+                    store_group(a.x + (size_t)i * a.ld, c, a.d, xn);
                 }
-                store_group(a.x + (size_t)i * a.ld, c, a.d, xn);
             }
         }
         if (it + 1 < my_tiles) {
@@ -175,49 +183,50 @@ int launch_halo(const dlm_shard_args& s, cudaStream_t stream) {
     const size_t tab = (size_t)(2 * s.n_loc + 1) * 4 + (size_t)s.nnz * 8;
     const int tables_in_smem = g_tune_tables == 1 ? 1 : g_tune_tables == 2 ? 0 : tab <= 8 * 1024;
     const size_t fixed = 128 + 16 + 16 + (tables_in_smem ? tab : 0);
-    // stage layout: x tile (own rows, gap up to n_pad, halo rows) | g tile (same rows) | m tile (own rows),
-    // every tile starting on a 128-byte boundary
+    // Stage layout: `boxes` x sub-tiles (own rows, gap up to n_pad, halo rows), then as many g sub-tiles
+    // (same rows), then the m sub-tiles (own rows); every sub-tile starts on a 128-byte boundary.
     auto align128 = [](size_t b) { return (b + 127) & ~(size_t)127; };
-    auto offsets_for = [&](int C, size_t& g_off, size_t& m_off) {
-        g_off = align128((size_t)rows * C * 4);
-        m_off = LAM ? align128(g_off + (size_t)rows * C * sizeof(GT)) : g_off;
-        return LAM ? align128(m_off + (size_t)s.n_loc * C * 4) : g_off;
-    };
     auto stage_bytes_for = [&](int C) {
-        size_t g_off, m_off;
-        return offsets_for(C, g_off, m_off);
+        const int Cb = std::min(C, 256), boxes = C / Cb;
+        size_t b = boxes * align128((size_t)rows * Cb * 4);
+        if (LAM) b += boxes * (align128((size_t)rows * Cb * sizeof(GT)) + align128((size_t)s.n_loc * Cb * 4));
+        return b;
     };
-    // Tile width: about 16 KB of staged x like the unsharded kernel, row segments of 128 bytes at
-    // least, and narrow enough for two CTAs per SM.
+    // Tile width: about 16 KB of staged x like the unsharded kernel (few rows: several 256-column boxes
+    // per tile), row segments of 128 bytes at least, and narrow enough for two CTAs per SM.
     int C = 1 << ilog2(std::max(1, (int)(16384 / ((size_t)rows * 4))));
-    C = std::max(32, std::min(256, C));
-    if (g_tune_cols >= 32 && g_tune_cols <= 256 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
+    C = std::max(32, std::min(2048, C));
+    if (g_tune_cols >= 32 && g_tune_cols <= 4096 && (g_tune_cols & (g_tune_cols - 1)) == 0) C = g_tune_cols;
     while (C > 32 && fixed + stage_bytes_for(C) > (size_t)dev.smem_optin / 2 - 1024) C /= 2;
     if (fixed + stage_bytes_for(C) > (size_t)dev.smem_optin) return DLM_ERR_UNSUPPORTED;
 
     HaloGeom geo;
     geo.C = C;
-    geo.cv_shift = ilog2(C / 4);
+    geo.box_cols = std::min(C, 256);
+    geo.boxes = C / geo.box_cols;
+    geo.cv_shift = ilog2(geo.box_cols / 4);
     geo.tables_in_smem = tables_in_smem;
-    geo.halo_x_off = (uint32_t)((size_t)s.n_pad * C * 4);            // n_pad even, C >= 32: 128-byte multiples
-    geo.halo_g_off = (uint32_t)((size_t)s.n_pad * C * sizeof(GT));
-    size_t g_off, m_off;
-    geo.stage_bytes = (uint32_t)offsets_for(C, g_off, m_off);
-    geo.g_off = (uint32_t)g_off;
-    geo.m_off = (uint32_t)m_off;
+    geo.sub_x = (uint32_t)align128((size_t)rows * geo.box_cols * 4);
+    geo.sub_g = LAM ? (uint32_t)align128((size_t)rows * geo.box_cols * sizeof(GT)) : 0u;
+    geo.sub_m = LAM ? (uint32_t)align128((size_t)s.n_loc * geo.box_cols * 4) : 0u;
+    geo.halo_x_off = (uint32_t)((size_t)s.n_pad * geo.box_cols * 4);  // n_pad even, box_cols >= 32: 128-byte multiples
+    geo.halo_g_off = (uint32_t)((size_t)s.n_pad * geo.box_cols * sizeof(GT));
+    geo.g_off = (uint32_t)geo.boxes * geo.sub_x;
+    geo.m_off = geo.g_off + (uint32_t)geo.boxes * geo.sub_g;
+    geo.stage_bytes = (uint32_t)stage_bytes_for(C);
     geo.tx_bytes = (uint32_t)((size_t)(s.n_loc + s.halo) * C * 4);
     if (LAM) geo.tx_bytes += (uint32_t)((size_t)(s.n_loc + s.halo) * C * sizeof(GT) + (size_t)s.n_loc * C * 4);
     geo.num_tiles = (s.d + C - 1) / C;
 
     CUtensorMap tm_x, tm_hx, tm_g, tm_hg, tm_m;
-    if (!make_map(&tm_x, s.x, false, s.n_loc, s.d, s.ld, C)) return DLM_ERR_UNSUPPORTED;
+    if (!make_map(&tm_x, s.x, false, s.n_loc, s.d, s.ld, geo.box_cols)) return DLM_ERR_UNSUPPORTED;
     // unused maps (no halo in this slot; no g, m for the averaging rule) alias the x map: never dereferenced
     tm_hx = tm_g = tm_hg = tm_m = tm_x;
-    if (s.halo > 0 && !make_map(&tm_hx, s.halo_x, false, s.halo, s.d, s.ld_halo_x, C)) return DLM_ERR_UNSUPPORTED;
+    if (s.halo > 0 && !make_map(&tm_hx, s.halo_x, false, s.halo, s.d, s.ld_halo_x, geo.box_cols)) return DLM_ERR_UNSUPPORTED;
     if (LAM) {
-        if (!make_map(&tm_g, s.g, bf16, s.n_loc, s.d, s.ldg, C) || !make_map(&tm_m, s.m, false, s.n_loc, s.d, s.ld, C))
+        if (!make_map(&tm_g, s.g, bf16, s.n_loc, s.d, s.ldg, geo.box_cols) || !make_map(&tm_m, s.m, false, s.n_loc, s.d, s.ld, geo.box_cols))
             return DLM_ERR_UNSUPPORTED;
-        if (s.halo > 0 && !make_map(&tm_hg, s.halo_g, bf16, s.halo, s.d, s.ld_halo_g, C)) return DLM_ERR_UNSUPPORTED;
+        if (s.halo > 0 && !make_map(&tm_hg, s.halo_g, bf16, s.halo, s.d, s.ld_halo_g, geo.box_cols)) return DLM_ERR_UNSUPPORTED;
     }
     dlm_step_args a = {};
     a.n = s.n_loc;
