@@ -201,7 +201,8 @@ DLM_API int dmsgd_step(const dlm_topology* topo, int64_t k, int n, int64_t d, in
  * place, there is no m; traffic is x and g read once, x written once (12 bytes per node-parameter).
  *   variant DLM_DSGD_ATC  adapt-then-combine, the DSGD of Sec. 3:  y_i = x_i - gamma g_i ;
  *                         x_i <- y_i + sum_{j != i} w_ij (y_j - y_i)            (= W (x - gamma g))
- *                         (bitwise the x that dmsgd_step gives with beta = 0)
+ *                         (the x that dmsgd_step gives with beta = 0: bit for bit when both calls take the
+ *                         same mixing kernel, see dlm_set_tuning knob 7, else to rounding)
  *   variant DLM_DSGD_AWC  adapt-with-combine of the Remark in Sec. 5:
  *                         x_i <- x_i + sum_{j != i} w_ij (x_j - x_i) - gamma g_i  (= W x - gamma g)
  * Other arguments and errors as for decentlam_step (no beta; DLM_ERR_KIND for an unknown variant).

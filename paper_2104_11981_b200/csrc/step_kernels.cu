@@ -434,14 +434,24 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     // single array either way and gains from the merged pass already at 8 entries per row.
     bool want_merged = a.max_degree >= 12 || (a.max_degree >= 8 && a.n <= 128);
     if (a.n > 128 && (long long)a.nnz < 8LL * a.n) want_merged = false;
-    // DecentLaM with compact tables (2-byte entries, three CTAs per SM at 256 nodes): ahead of the plain loop
-    // from 8 entries per row on at every size measured (static exponential graph of 256 nodes +10 %,
-    // Erdos-Renyi graphs +25 to +40 %), level with it at 7 (exponential graph of 64 nodes), behind at 3 .. 6
-    if (RULE == DLM_RULE_DECENTLAM && a.compact) want_merged = a.max_degree >= 8;
     if (RULE == DLM_RULE_DMSGD) want_merged = a.max_degree >= 8;
     // one staged array and no momentum in pass 2: up to 128 nodes DmSGD and adapt-then-combine DSGD gain
     // 1 to 7 % from six entries per row on (exponential graphs of 32 and 64 nodes)
     if ((RULE == DLM_RULE_DMSGD || RULE == DLM_RULE_DSGD_ATC) && a.n <= 128 && a.max_degree >= 6) want_merged = true;
+    // With compact tables (2-byte entries; built-in graphs and Metropolis-Hastings weights up to 256 nodes)
+    // the merged kernel is ahead much earlier, measured on 409 M node-parameters:
+    //   DecentLaM  from 8 entries per row on (static exponential graph of 256 nodes +10 %, Erdos-Renyi graphs
+    //              +25 to +40 %); level at 7 (exponential graph of 64 nodes), behind at 2 .. 6
+    //   DmSGD      from 64 nodes on whatever the rows (rings of 64 / 128 / 256 nodes +10 / +6 / +20 %), and from 6
+    //              entries per row on below that
+    //   DSGD       from 32 nodes on (rings, one-peer, mesh: +3 to +15 %); from 12 nodes on for
+    //              adapt-then-combine (+3 to +15 %) and, with three or more entries per row, for adapt-with-combine
+    if (a.compact) {
+        if (RULE == DLM_RULE_DECENTLAM) want_merged = a.max_degree >= 8;
+        if (RULE == DLM_RULE_DMSGD) want_merged = a.n >= 64 || a.max_degree >= 6;
+        if (RULE == DLM_RULE_DSGD_ATC) want_merged = a.n >= 12;
+        if (RULE == DLM_RULE_DSGD_AWC) want_merged = a.n >= 32 || (a.n >= 12 && a.max_degree >= 3);
+    }
     const bool merged = (g_tune_mix == 2 || g_tune_mix == 3) ? true : g_tune_mix == 1 ? false : want_merged;
     if (merged) {
         int rc = dlm_launch_merged(RULE, a, stream);

@@ -309,8 +309,8 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Compact-table form of the merged DecentLaM kernel (same staging, same pass 1, same sums up to the
-// position of the self term).  What differs is how pass 2 learns its neighbours:
+// Compact-table form of the merged kernel, all four rules (same staging, same pass 1, same sums up to
+// the position of the self term).  What differs is how pass 2 learns its neighbours:
 //   * the tables are packed (4 bytes per row, 2 bytes per off-diagonal entry: {column, index into a
 //     small table of the distinct weights}), about a third of the 8-byte entries' size, so that a
 //     third CTA fits beside two others in an SM's shared memory at 256 nodes;
@@ -318,17 +318,19 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
 //     address: a broadcast), instead of fetching them four at a time and handing them round with
 //     two shuffles per entry, which occupy the same data pipe as the shared-memory loads;
 //   * the loop ends at the longest row of the warp, not at the next multiple of four.
-// The self term w_ii v_i is added after the loop from a per-row weight (diagonal weights are
-// remainders 1 - sum and rarely repeat, so they would not fit a small table).
+// The self term is added after the loop from a per-row weight (diagonal weights are remainders
+// 1 - sum and rarely repeat, so they would not fit a small table): the stored w_ii for DecentLaM's
+// v-sum, the exact remainder 1 - sum_{j != i} w_ij (a.selfw) for the averaging rules.
 // Available when the slot has at most 256 nodes, 255 distinct off-diagonal weights and 65535
 // off-diagonal entries (Metropolis-Hastings and all built-in graphs: a few dozen weights).
 // Blob layout (a.compact): rowrec u32[n] {i | len << 8 | first << 16} in processing order, S f32[n],
 // wself f32[n], wlut f32[nw + 1] (last = 0, the filler's weight), cent u16[noff] {col | widx << 8}.
 // ---------------------------------------------------------------------------------------------
-template <typename GT, int THREADS, int MIN_CTAS>
+template <int RULE, typename GT, int THREADS, int MIN_CTAS>
 __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                                          const __grid_constant__ CUtensorMap tm_g,
                                                                          dlm_step_args a, MergedGeom geo) {
+    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char* st = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
     uint64_t* bar_ptr = reinterpret_cast<uint64_t*>(st + geo.stage_bytes);
@@ -363,7 +365,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
     __syncthreads();
 
     float* xs = reinterpret_cast<float*>(st);
-    float* vs = reinterpret_cast<float*>(st + geo.v_off);
+    float* vs = reinterpret_cast<float*>(st + geo.v_off);  // staged values: v (DecentLaM) or y (the x tile itself)
     const GT* gs = reinterpret_cast<const GT*>(st + geo.g_off);
     const int items = a.n << geo.cv_shift;
     const int cv_mask = (1 << geo.cv_shift) - 1;
@@ -377,9 +379,22 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
     const int row_shift = geo.cv_shift + 4;  // log2 of the row pitch in bytes (C * 4)
     const uint32_t filler_w = (uint32_t)a.compact_nw << 8;
 
+    // DmSGD: pass-1 items per thread whose m is fetched before the wait for the tile (all of them at 256 and
+    // at 512 threads for tiles of 8192 elements)
+    constexpr int kPre = THREADS >= 384 ? 4 : 8;
     for (long long it = 0; it < my_tiles; ++it) {
         const long long tile_base = (first_tile + it * gridDim.x) * C;
-        if (geo.prefetch_m) {
+        Pack<4> mpre[kPre];
+        if (RULE == DLM_RULE_DMSGD) {  // m straight from global memory, in flight while the tile lands
+#pragma unroll
+            for (int k = 0; k < kPre; ++k) {
+                const int e = threadIdx.x + k * THREADS;
+                const long long c = tile_base + (e & cv_mask) * 4;
+                mpre[k] = {{0.f, 0.f, 0.f, 0.f}};
+                if (e < items && c < a.d) mpre[k] = ld_f32<4>(a.m + (size_t)(e >> geo.cv_shift) * a.ld + c);
+            }
+        }
+        if (LAM && geo.prefetch_m) {
             const int seg_shift = geo.cv_shift - 3, segs = a.n << seg_shift;  // C / 32 segments per row
             for (int e = threadIdx.x; e < 2 * segs; e += THREADS) {
                 const int sg = e >> 1;
@@ -395,18 +410,40 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
             __syncthreads();
             return;
         }
-        // pass 1: v = g - (x - r) / gamma, r = row 0's value of the column
-        for (int e = threadIdx.x; e < items; e += THREADS) {
-            const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
-            const Pack<4> xi = ld_f32<4>(xs + i * C + off);
-            const Pack<4> gi = ld_g<4>(gs + i * C + off);
-            const Pack<4> ref = ld_f32<4>(xs + off);
-            Pack<4> v;
+        // pass 1.  DecentLaM: v = g - (x - r) / gamma, r = row 0's value of the column.  DmSGD: m' = beta m + g,
+        // y = x - gamma m'.  Adapt-then-combine: y = x - gamma g.  Adapt-with-combine averages x as it is.
+        if (RULE != DLM_RULE_DSGD_AWC) {
+            int k = 0;
+            for (int e = threadIdx.x; e < items; e += THREADS, ++k) {
+                const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+                const Pack<4> xi = ld_f32<4>(xs + i * C + off);
+                const Pack<4> gi = ld_g<4>(gs + i * C + off);
+                Pack<4> v;
+                if (LAM) {
+                    const Pack<4> ref = ld_f32<4>(xs + off);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
-            st_f32<4>(vs + i * C + off, v);
+                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi.v[u]);
+                } else if (RULE == DLM_RULE_DMSGD) {
+                    const long long c = tile_base + off;
+                    Pack<4> mi = {{0.f, 0.f, 0.f, 0.f}}, mn;
+                    if (k < kPre) {
+#pragma unroll
+                        for (int q = 0; q < kPre; ++q)
+                            if (q == k) mi = mpre[q];
+                    } else if (c < a.d) {
+                        mi = ld_f32<4>(a.m + (size_t)i * a.ld + c);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) dmsgd_local(xi.v[u], mi.v[u], gi.v[u], a.beta, a.gamma, mn.v[u], v.v[u]);
+                    if (c < a.d) st_f32<4>(a.m + (size_t)i * a.ld + c, mn);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.gamma, gi.v[u], xi.v[u]);
+                }
+                st_f32<4>(vs + i * C + off, v);
+            }
+            __syncthreads();
         }
-        __syncthreads();
         // pass 2
         // Rows come in order of decreasing length, one warp-load of 32 / L rows after the other.  The warps
         // take these loads boustrophedon (warp w: load w, then 2W-1-w, then 2W+w, ...), so that every
@@ -428,8 +465,10 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
             const long long c0 = tile_base + off0, c1 = tile_base + off1;
             const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;
             Pack<4> m0 = {{0.f, 0.f, 0.f, 0.f}}, m1 = {{0.f, 0.f, 0.f, 0.f}};
-            if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
-            if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            if (LAM) {
+                if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
+                if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            }
             float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t vb0 = smem_u32(vs) + off0 * 4, vb1 = smem_u32(vs) + off1 * 4;
             const uint32_t filler = (uint32_t)i | filler_w;  // adds exactly 0 * (staged value of row i)
@@ -448,23 +487,35 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
                 acc1[0] = fmaf(w, v1.x, acc1[0]); acc1[1] = fmaf(w, v1.y, acc1[1]);
                 acc1[2] = fmaf(w, v1.z, acc1[2]); acc1[3] = fmaf(w, v1.w, acc1[3]);
             }
-            const float S_i = Ssum[slot], w_ii = wself[slot];
+            // self weight: the stored diagonal for DecentLaM's v-sum, the exact remainder for the averages
+            const float S_i = LAM ? Ssum[slot] : 0.f;
+            const float w_ii = LAM ? wself[slot] : (live ? __int_as_float(a.selfw[slot]) : 0.f);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int off = h ? off1 : off0;
-                const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off), vi = ld_f32<4>(vs + i * C + off);
-                Pack<4> mn, xn;
+                const Pack<4> vi = ld_f32<4>(vs + i * C + off);
+                Pack<4> xn;
+                if (LAM) {
+                    const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
+                    Pack<4> mn;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float mix = fmaf(w_ii, vi.v[u], h ? acc1[u] : acc0[u]);  // self term of the v-sum
-                    const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, mix);
-                    mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
-                    xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
+                    for (int u = 0; u < 4; ++u) {
+                        const float mix = fmaf(w_ii, vi.v[u], h ? acc1[u] : acc0[u]);  // self term of the v-sum
+                        const float gt = fmaf((xi.v[u] - ref.v[u]) * S_i, a.inv_gamma, mix);
+                        mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
+                        xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
+                    }
+                    if (h ? st1 : st0) st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(w_ii, vi.v[u], h ? acc1[u] : acc0[u]);
+                    if (RULE == DLM_RULE_DSGD_AWC) {
+                        const Pack<4> gi = ld_g<4>(gs + i * C + off);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
+                    }
                 }
-                if (h ? st1 : st0) {
-                    st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
-                    st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
-                }
+                if (h ? st1 : st0) st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
             }
         }
         if (it + 1 < my_tiles) {
@@ -477,10 +528,11 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
 
 int g_tune_compact_threads = 0;  // knob 12: block size of the compact-table kernel (256, 384 or 512), 0 = auto
 
-// Compact-table merged kernel (DecentLaM).  DLM_ERR_UNSUPPORTED if the slot has no compact tables or the
-// shape does not fit.
-template <typename GT>
+// Compact-table merged kernel.  DLM_ERR_UNSUPPORTED if the slot has no compact tables or the shape does
+// not fit.
+template <int RULE, typename GT>
 int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
+    constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
     const DeviceInfo& dev = device_info();
     if (!dev.ok) return DLM_ERR_CUDA;
     const bool bf16 = sizeof(GT) == 2;
@@ -496,9 +548,15 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
         const size_t xb = ((size_t)a.n * C * 4 + 127) & ~(size_t)127;
         const size_t gb = ((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127;
         geo.x_bytes = (uint32_t)xb;
-        geo.v_off = (uint32_t)xb;   // [x | v | g]: for fp32 gradients v overwrites g in place
-        geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);
-        geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
+        if (LAM) {  // [x | v | g]: for fp32 gradients v overwrites g in place
+            geo.v_off = (uint32_t)xb;
+            geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);
+            geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
+        } else {    // [x (becomes y) | g]
+            geo.v_off = 0;
+            geo.g_off = (uint32_t)xb;
+            geo.stage_bytes = (uint32_t)(xb + gb);
+        }
         smem = 128 + 16 + geo.stage_bytes + (size_t)a.compact_bytes;
         if (2 * (smem + 1024) <= sm_total || (C == 32 && smem <= (size_t)dev.smem_optin)) break;
     }
@@ -514,15 +572,22 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : 4;
     const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
     const bool three = 3 * (smem + 1024) <= sm_total;
-    // Block size (measured on Erdos-Renyi, exponential and complete graphs of 16 .. 256 nodes): few, fat
-    // threads win where tiles are narrow (n >= 128, fp32: 128 threads beat 256 by 5 to 7 %, 512 lose 10 %);
-    // up to 64 nodes and with bf16 gradients 256 threads are 2 to 10 % ahead.
+    // Block size, measured on ring, exponential, Erdos-Renyi and complete graphs of 8 .. 256 nodes.
+    //   DecentLaM: few, fat threads win where tiles are narrow (n >= 128, fp32: 128 threads beat 256 by 5 to
+    //     7 %, 512 lose 10 %); up to 64 nodes and with bf16 gradients 256 threads are 2 to 10 % ahead.
+    //   DmSGD reads m in pass 1 from global memory: only with 512 threads are all of those loads issued
+    //     before the wait for the tile (256 threads: 10 to 15 % slower, 128: 40 %).
+    //   DSGD (no momentum, the lightest pass 2): 256 threads, three CTAs per SM.
+    //   Up to 16 nodes (tiles of 256 columns, a warp per row): 128 threads for every rule.
     int threads = g_tune_compact_threads;
-    if (threads != 128 && threads != 256 && threads != 384 && threads != 512)
-        threads = (!bf16 && (a.n >= 128 || a.n <= 16)) ? 128 : 256;
+    if (threads != 128 && threads != 256 && threads != 384 && threads != 512) {
+        if (a.n <= 16) threads = 128;
+        else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;
+        else threads = RULE == DLM_RULE_DMSGD ? 512 : 256;
+    }
 #define DLM_COMPACT_LAUNCH(T, M)                                                                               \
     {                                                                                                          \
-        auto kern = step_compact_kernel<GT, T, M>;                                                             \
+        auto kern = step_compact_kernel<RULE, GT, T, M>;                                                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
             return DLM_ERR_CUDA;                                                                               \
         kern<<<(unsigned)grid, T, smem, stream>>>(tm_x, tm_g, a, geo);                                         \
@@ -549,18 +614,19 @@ int dlm_launch_merged(int rule, const dlm_step_args& a, void* stream) {
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const bool bf16 = a.g_dtype == DLM_G_BF16;
     switch (rule) {
-    case DLM_RULE_DECENTLAM:
-        if (g_tune_mix != 2) {  // compact-table form wherever the slot has compact tables (knob 7 = 2: the 8-byte entries)
-            const int rc = bf16 ? launch_compact<__nv_bfloat16>(a, s) : launch_compact<float>(a, s);
-            if (rc != DLM_ERR_UNSUPPORTED) return rc;
-        }
-        return bf16 ? launch_merged<DLM_RULE_DECENTLAM, __nv_bfloat16>(a, s) : launch_merged<DLM_RULE_DECENTLAM, float>(a, s);
-    case DLM_RULE_DMSGD:
-        return bf16 ? launch_merged<DLM_RULE_DMSGD, __nv_bfloat16>(a, s) : launch_merged<DLM_RULE_DMSGD, float>(a, s);
-    case DLM_RULE_DSGD_ATC:
-        return bf16 ? launch_merged<DLM_RULE_DSGD_ATC, __nv_bfloat16>(a, s) : launch_merged<DLM_RULE_DSGD_ATC, float>(a, s);
-    case DLM_RULE_DSGD_AWC:
-        return bf16 ? launch_merged<DLM_RULE_DSGD_AWC, __nv_bfloat16>(a, s) : launch_merged<DLM_RULE_DSGD_AWC, float>(a, s);
+#define DLM_MERGED_RULE(R)                                                                                   \
+    case R: {                                                                                                \
+        if (g_tune_mix != 2) { /* compact tables where the slot has them (knob 7 = 2: the 8-byte entries) */ \
+            const int rc = bf16 ? launch_compact<R, __nv_bfloat16>(a, s) : launch_compact<R, float>(a, s);   \
+            if (rc != DLM_ERR_UNSUPPORTED) return rc;                                                        \
+        }                                                                                                    \
+        return bf16 ? launch_merged<R, __nv_bfloat16>(a, s) : launch_merged<R, float>(a, s);                 \
+    }
+        DLM_MERGED_RULE(DLM_RULE_DECENTLAM)
+        DLM_MERGED_RULE(DLM_RULE_DMSGD)
+        DLM_MERGED_RULE(DLM_RULE_DSGD_ATC)
+        DLM_MERGED_RULE(DLM_RULE_DSGD_AWC)
+#undef DLM_MERGED_RULE
     default:
         return DLM_ERR_KIND;
     }

@@ -39,13 +39,24 @@ def test_dsgd_matches_oracle(rule, topology, n, d, g_dtype):
     assert rel_l2(to64(x), xo) <= TOL_T
 
 
-def test_atc_is_bitwise_dmsgd_with_beta_zero():
+def test_atc_is_dmsgd_with_beta_zero():
+    """Adapt-then-combine DSGD is DmSGD with beta = 0: bit for bit when both take the same kernel path (forced
+    here to the plain mixing loop), to rounding when the automatic choice sends them different ways."""
     dev = torch.device("cuda:0")
     from paper_2104_11981_b200 import binding as B
-    for n, d, topology in ((16, 200_000, "one_peer_exp"), (8, 1000, "ring")):
+    for n, d, topology in ((16, 200_000, "one_peer_exp"), (8, 1000, "ring"), (64, 50_000, "static_exp")):
         topo, _ = build_both(topology, n)
         x0 = inputs.normal_torch((n, d), 0.02, 3, dev); g = inputs.normal_torch((n, d), 1e-3, 4, dev)
-        xa = x0.clone(); B.dsgd_step(topo, 1, xa, g, 0.1, B.DSGD_ATC)
-        xb = x0.clone(); mb = torch.zeros_like(xb); B.dmsgd_step(topo, 1, xb, mb, g, 0.0, 0.1)
-        torch.cuda.synchronize()
-        assert torch.equal(xa, xb) and torch.equal(mb, g)
+        for mix in (1, 0):
+            try:
+                B.set_tuning(7, mix)
+                xa = x0.clone(); B.dsgd_step(topo, 1, xa, g, 0.1, B.DSGD_ATC)
+                xb = x0.clone(); mb = torch.zeros_like(xb); B.dmsgd_step(topo, 1, xb, mb, g, 0.0, 0.1)
+                torch.cuda.synchronize()
+            finally:
+                B.set_tuning(7, 0)
+            assert torch.equal(mb, g)
+            if mix == 1:
+                assert torch.equal(xa, xb)
+            else:
+                assert rel_l2(to64(xa), to64(xb)) <= 1e-6

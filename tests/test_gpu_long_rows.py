@@ -31,20 +31,21 @@ def test_long_rows_sampled(topology, n, er_p, d, rule, g_dtype):
     _run(topology, n, er_p, d, rule, g_dtype)
 
 
-@pytest.mark.parametrize("threads", [128, 256, 384, 512])
+@pytest.mark.parametrize("rule,threads", [("decentlam", 128), ("decentlam", 256), ("decentlam", 384), ("decentlam", 512),
+                                          ("dmsgd", 128), ("dmsgd", 512), ("dsgd_atc", 256), ("dsgd_awc", 128), ("dsgd_awc", 384)])
 @pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("topology,n,er_p,d", SHAPES + [("er_mh", 256, 0.05, 300_008), ("ring", 200, 0.0, 200_008)])
-def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, threads):
-    """The compact-table form of the merged DecentLaM kernel (2-byte entries, per-lane entry loads, self term
+def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, rule, threads):
+    """The compact-table form of the merged kernel (2-byte entries, per-lane entry loads, self term
     added last, rows dealt to the warps boustrophedon), forced by knob 7 = 3 at each of its block sizes; and the
     older form with 8-byte entries and shuffles (knob 7 = 2), which general weight tables still take."""
     from paper_2104_11981_b200 import binding as B
     try:
         B.set_tuning(7, 3); B.set_tuning(12, threads)
-        _run(topology, n, er_p, d, "decentlam", g_dtype)
+        _run(topology, n, er_p, d, rule, g_dtype)
         if threads == 512:
             B.set_tuning(7, 2)
-            _run(topology, n, er_p, d, "decentlam", g_dtype)
+            _run(topology, n, er_p, d, rule, g_dtype)
     finally:
         B.set_tuning(7, 0); B.set_tuning(12, 0)
 
