@@ -559,6 +559,9 @@ def run_sharded(args):
     n, d = w.n, (args.columns or w.d)
     gdt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
     topo = build_topology(B, inputs, args.workload)
+    for item in filter(None, args.tuning.split(",")):
+        knob, value = item.split("=")
+        B.set_tuning(int(knob), int(value))
     shard = B.topology_shard(topo, rank if world > 1 else 0, ranks)
     lo, hi, max_halo = shard.rows
     n_loc = hi - lo

@@ -254,8 +254,13 @@ int launch_halo(const dlm_shard_args& s, cudaStream_t stream) {
         return DLM_ERR_CUDA;
     const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : (tab <= 2560 ? 1 : 4);
     const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    // Block size by the mixing work of a tile (own rows x longest row), measured on the three large
+    // workloads cut into 2 .. 16 ranks: 128 threads up to 512 row-entries (1 to 16 own rows of any graph
+    // measured: +5 to +45 % over 256 threads, several more CTAs per SM overlap their copies), 256 up to 1024
+    // (32 own rows of 14 entries), 512 beyond (64 and 128 own rows of 14 entries).
+    const long long work = (long long)s.n_loc * s.max_degree;
     const int threads = (g_tune_threads == 128 || g_tune_threads == 256 || g_tune_threads == 512)
-                            ? g_tune_threads : (s.max_degree > 8 ? 512 : 256);
+                            ? g_tune_threads : (work >= 1024 ? 512 : work >= 512 ? 256 : 128);
     kern<<<(unsigned)grid, threads, smem, stream>>>(tm_x, tm_hx, tm_g, tm_hg, tm_m, a, s.halo, geo);
     dlm_count_launch(1);
     return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
