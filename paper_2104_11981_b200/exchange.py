@@ -19,12 +19,31 @@ def _runs(dst_slots):
     return runs
 
 
-def post_halo_exchange(dist, shard, slot, arrays, halos, group=None):
-    """Post the sends and receives of one slot for several arrays at once and wait for them.
+class PendingExchange:
+    """The transfers of one posted exchange: `wait()` blocks (the current stream, for NCCL) until this
+    rank's receives have landed and its send buffers may be overwritten."""
 
-    arrays : list of tensors [n_loc, d] holding the rank's own rows (e.g. [x, g]); rows must be contiguous
-    halos  : list of tensors [>= halo, d], same dtypes, contiguous: halos[a][t] receives row rows[t] of array a
-    Returns the number of bytes this rank received.
+    def __init__(self, requests, keep, received):
+        self.requests, self.keep, self.received = requests, keep, received
+
+    def wait(self):
+        for req in self.requests:
+            req.wait()
+        self.requests, self.keep = [], []
+        return self.received
+
+
+def post_halo_exchange(dist, shard, slot, arrays, halos, group=None, cols=None, wait=True):
+    """Post the sends and receives of one slot for several arrays at once.
+
+    arrays : list of tensors [n_loc, d] holding the rank's own rows (e.g. [x, g]), unit column stride
+    halos  : list of contiguous tensors, same dtypes: halos[a][t] receives row rows[t] of array a.
+             Whole rows: [>= halo, d].  With cols = (c0, c1): [>= halo, c1 - c0], the buffer of that
+             column chunk alone (the kernel is then called on the chunk with this buffer as its halo).
+    cols   : column range to exchange, or None for whole rows; a chunk of the own rows is packed into a
+             contiguous send buffer first (a slice of a row-major array is not contiguous)
+    wait   : True: wait for the transfers and return the number of bytes received.  False: return a
+             PendingExchange at once, so that the caller can run the previous chunk's kernel meanwhile.
     """
     import torch
     rank, world = dist.get_rank(group), dist.get_world_size(group)
@@ -37,10 +56,15 @@ def post_halo_exchange(dist, shard, slot, arrays, halos, group=None):
         rows, _ = shard.sends(slot, peer)
         if len(rows):
             local = torch.as_tensor(rows - row_lo, dtype=torch.long, device=arrays[0].device)
-            contiguous = bool(rows[-1] - rows[0] + 1 == len(rows))
+            first = int(rows[0] - row_lo)
+            consecutive = bool(rows[-1] - rows[0] + 1 == len(rows))
             for a in arrays:
-                # consecutive own rows go out as a view; a scattered set is packed into one buffer first
-                buf = a[int(local[0]): int(local[0]) + len(rows)] if contiguous else a.index_select(0, local)
+                # consecutive own rows go out as a view when that view is contiguous; a scattered set, or a
+                # column chunk, is packed into one buffer first
+                src = a[first: first + len(rows)] if consecutive else a.index_select(0, local)
+                if cols is not None:
+                    src = src[:, cols[0]: cols[1]]
+                buf = src if src.is_contiguous() else src.contiguous()
                 keep.append(buf)
                 ops.append(dist.P2POp(dist.isend, buf, peer, group))
         mine = [t for t in range(len(halo_rows)) if owners[t] == peer]
@@ -50,12 +74,18 @@ def post_halo_exchange(dist, shard, slot, arrays, halos, group=None):
             assert mine[-1] - t0 + 1 == cnt
             for h in halos:
                 slab = h[t0: t0 + cnt]
+                assert slab.is_contiguous()
                 received += slab.numel() * slab.element_size()
                 ops.append(dist.P2POp(dist.irecv, slab, peer, group))
-    if ops:
-        for req in dist.batch_isend_irecv(ops):
-            req.wait()
-    return received
+    pending = PendingExchange(dist.batch_isend_irecv(ops) if ops else [], keep, received)
+    return pending.wait() if wait else pending
+
+
+def column_chunks(d, chunk_cols):
+    """Column ranges [(c0, c1), ...] of width chunk_cols (a multiple of 8, so that every chunk of a 16-byte
+    aligned row starts 16-byte aligned for fp32 and bf16 alike); the last one may be narrower."""
+    assert chunk_cols >= 8 and chunk_cols % 8 == 0
+    return [(c0, min(d, c0 + chunk_cols)) for c0 in range(0, d, chunk_cols)]
 
 
 def halo_bytes_per_step(shard, slot, d, bytes_per_row_element):

@@ -112,6 +112,37 @@ def test_sharded_step_against_the_oracle(rule):
     assert B.kernel_error() == 0
 
 
+def test_sharded_step_in_column_chunks_is_bitwise_the_whole_step():
+    """The pipelined form of a sharded run exchanges and updates the columns chunk by chunk, each chunk with a
+    halo buffer of its own (row stride = chunk width) and column-sliced views of the own rows: bit for bit the
+    step on whole rows, because every rule is coordinate-wise."""
+    from paper_2104_11981_b200 import binding as B
+    from paper_2104_11981_b200 import exchange
+    dev = torch.device("cuda:0")
+    n, d, ranks = 16, 50_024, 4
+    topo, _ = build_both("one_peer_exp", n)
+    shards = [B.topology_shard(topo, r, ranks) for r in range(ranks)]
+    x = inputs.normal_torch((n, d), 0.02, 31, dev); m = inputs.normal_torch((n, d), 0.01, 32, dev)
+    g = inputs.normal_torch((n, d), 1e-3, 33, dev)
+    for k in range(4):
+        want_x, want_m = _sharded_step(B, "decentlam", shards, k, x, m, g, 0.9, 0.1)
+        got_x, got_m = torch.empty_like(x), torch.empty_like(m)
+        for sh in shards:
+            lo, hi, _ = sh.rows
+            rows, _ = sh.halo(k % topo.period)
+            idx = torch.as_tensor(rows, dtype=torch.long, device=dev)
+            xr, mr, gr = x[lo:hi].clone(), m[lo:hi].clone(), g[lo:hi].clone()
+            for c0, c1 in exchange.column_chunks(d, 16_384):
+                hx = x.index_select(0, idx)[:, c0:c1].contiguous()
+                hg = g.index_select(0, idx)[:, c0:c1].contiguous()
+                B.decentlam_step_sharded(sh, k, xr[:, c0:c1], mr[:, c0:c1], gr[:, c0:c1], hx, hg, 0.9, 0.1)
+            got_x[lo:hi], got_m[lo:hi] = xr, mr
+        torch.cuda.synchronize()
+        assert torch.equal(got_x, want_x) and torch.equal(got_m, want_m), k
+        x, m = want_x, want_m
+    assert B.kernel_error() == 0
+
+
 def test_sharded_step_argument_errors():
     from paper_2104_11981_b200 import binding as B
     import ctypes

@@ -115,6 +115,21 @@ for topology, n in {cases!r}:
         ok = bool(torch.equal(halo_x[:len(need)], want_x)) and bool(torch.equal(halo_g[:len(need)], (-want_x - 0.5).to(torch.bfloat16).float()))
         ok = ok and bool((halo_x[len(need):] == -7.0).all()) and got == 2 * len(need) * d * 4
         ok = ok and got == exchange.halo_bytes_per_step(sh, slot, d, 8)
+        # the same rows again as a pipelined exchange of column chunks: chunk j+1 is posted before chunk j is
+        # waited for, each chunk lands in a buffer of its own
+        chunks = exchange.column_chunks(d, 16)
+        bufs = [(torch.full((max(1, max_halo), c1 - c0), -7.0), torch.full((max(1, max_halo), c1 - c0), -7.0)) for c0, c1 in chunks]
+        pend = exchange.post_halo_exchange(dist, sh, slot, [own_x, own_g], list(bufs[0]), cols=chunks[0], wait=False)
+        got_chunks = 0
+        for j, (c0, c1) in enumerate(chunks):
+            nxt = None
+            if j + 1 < len(chunks):
+                nxt = exchange.post_halo_exchange(dist, sh, slot, [own_x, own_g], list(bufs[j + 1]), cols=chunks[j + 1], wait=False)
+            got_chunks += pend.wait()
+            ok = ok and bool(torch.equal(bufs[j][0][:len(need)], want_x[:, c0:c1])) and \
+                bool(torch.equal(bufs[j][1][:len(need)], (-want_x[:, c0:c1] - 0.5).to(torch.bfloat16).float()))
+            pend = nxt
+        ok = ok and got_chunks == got
         report.append([topology, n, slot, len(need), ok])
     dist.barrier()
 dist.destroy_process_group()
@@ -131,7 +146,8 @@ def _free_port():
 @pytest.mark.parametrize("world", [2, 4])
 def test_halo_exchange_delivers_the_referenced_rows_on_gloo_ranks(world):
     """world gloo ranks on the CPU run the exchange of every slot of several graphs: each rank must end
-    up with exactly the rows its block's weights reference, in ascending order, and nothing else."""
+    up with exactly the rows its block's weights reference, in ascending order, and nothing else; once as
+    whole rows, once as a pipeline of column chunks (the next chunk posted before the current one is waited for)."""
     port = _free_port()
     cases = [c for c in CASES if c[1] >= world]
     procs = []
