@@ -412,7 +412,7 @@ DLM_API int dlm_kernel_error(int* flag);
  *   knob 11 lsq_grad_gram: share of H kept in L2 with evict-last priority between calls, in 1/1000
  *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
  *           size, else none)
- *   knob 12 block size of the compact-table merged kernel (128, 256, 384 or 512)
+ *   knob 12 block size of the compact-table merged kernel (128, 256 or 512)
  * Results do not depend on the knobs, with one exception: the merged-staging kernels (knob 7 = 2 or 3,
  * the default on long rows: 8 or more entries; 12 or more for dsgd_step above 128 nodes) arrange the same
  * sum differently and agree with the other paths, and with each other, to rounding, not bitwise.

@@ -526,7 +526,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
     }
 }
 
-int g_tune_compact_threads = 0;  // knob 12: block size of the compact-table kernel (256, 384 or 512), 0 = auto
+int g_tune_compact_threads = 0;  // knob 12: block size of the compact-table kernel (128, 256 or 512), 0 = auto
 
 // Compact-table merged kernel.  DLM_ERR_UNSUPPORTED if the slot has no compact tables or the shape does
 // not fit.
@@ -571,7 +571,6 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
         return DLM_ERR_UNSUPPORTED;
     const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : 4;
     const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
-    const bool three = 3 * (smem + 1024) <= sm_total;
     // Block size, measured on ring, exponential, Erdos-Renyi and complete graphs of 8 .. 256 nodes.
     //   DecentLaM: few, fat threads win where tiles are narrow (n >= 128, fp32: 128 threads beat 256 by 5 to
     //     7 %, 512 lose 10 %); up to 64 nodes and with bf16 gradients 256 threads are 2 to 10 % ahead.
@@ -580,7 +579,7 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     //   DSGD (no momentum, the lightest pass 2): 256 threads, three CTAs per SM.
     //   Up to 16 nodes (tiles of 256 columns, a warp per row): 128 threads for every rule.
     int threads = g_tune_compact_threads;
-    if (threads != 128 && threads != 256 && threads != 384 && threads != 512) {
+    if (threads != 128 && threads != 256 && threads != 512) {
         if (a.n <= 16) threads = 128;
         else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;
         else threads = RULE == DLM_RULE_DMSGD ? 512 : 256;
@@ -594,8 +593,6 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     }
     if (threads == 128) DLM_COMPACT_LAUNCH(128, 3)
     else if (threads == 256) DLM_COMPACT_LAUNCH(256, 3)
-    else if (threads == 384 && three) DLM_COMPACT_LAUNCH(384, 3)
-    else if (threads == 384) DLM_COMPACT_LAUNCH(384, 2)
     else DLM_COMPACT_LAUNCH(512, 2)
 #undef DLM_COMPACT_LAUNCH
     dlm_count_launch(1);

@@ -115,6 +115,33 @@ def adjacency_to_lists(adj):
     return rowptr, (np.concatenate(cols) if cols else np.zeros(0, np.int32)).astype(np.int32)
 
 
+def random_doubly_stochastic(n, p, seed, iterations=2000):
+    """A general symmetric doubly-stochastic weight matrix on a connected Erdos-Renyi(p) graph with self
+    loops, as CSR (rowptr int32, col int32, val float32) plus the dense float64 matrix of those fp32 values.
+    Random positive weights on the pattern are balanced by symmetric diagonal scaling (W <- D W D with
+    D = diag(rowsum)^(-1/2), repeated in float64 until every row sums to one within 1e-12), then rounded
+    once to fp32: practically every entry is a different number, unlike the 1/q weights of the built-in
+    graphs.  Row and column sums of the fp32 values are within 1e-6 of one."""
+    adj, _ = er_adjacency(n, p, seed)
+    rng = np.random.Generator(np.random.Philox(seed + 1))
+    raw = rng.uniform(0.5, 1.5, size=(n, n))
+    W = np.where(adj > 0, (raw + raw.T) / 2, 0.0) + np.diag(rng.uniform(0.5, 1.5, size=n))
+    for _ in range(iterations):
+        r = W.sum(axis=1)
+        if np.max(np.abs(r - 1.0)) < 1e-12:
+            break
+        dinv = 1.0 / np.sqrt(r)
+        W = W * dinv[:, None] * dinv[None, :]
+    W32 = W.astype(np.float32)
+    rowptr = np.zeros(n + 1, dtype=np.int32)
+    cols, vals = [], []
+    for i in range(n):
+        nz = np.nonzero(W32[i])[0].astype(np.int32)
+        cols.append(nz); vals.append(W32[i, nz])
+        rowptr[i + 1] = rowptr[i] + len(nz)
+    return rowptr, np.concatenate(cols).astype(np.int32), np.concatenate(vals).astype(np.float32), W32.astype(np.float64)
+
+
 def bipartite_matchings(n, period, seed):
     """`period` random perfect matchings of n nodes (n even), one per iteration, as App. G's
     "bipartite random match": the nodes are split at random into two halves and paired.

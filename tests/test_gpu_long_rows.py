@@ -31,8 +31,8 @@ def test_long_rows_sampled(topology, n, er_p, d, rule, g_dtype):
     _run(topology, n, er_p, d, rule, g_dtype)
 
 
-@pytest.mark.parametrize("rule,threads", [("decentlam", 128), ("decentlam", 256), ("decentlam", 384), ("decentlam", 512),
-                                          ("dmsgd", 128), ("dmsgd", 512), ("dsgd_atc", 256), ("dsgd_awc", 128), ("dsgd_awc", 384)])
+@pytest.mark.parametrize("rule,threads", [("decentlam", 128), ("decentlam", 256), ("decentlam", 512), ("dmsgd", 128),
+                                          ("dmsgd", 256), ("dmsgd", 512), ("dsgd_atc", 256), ("dsgd_awc", 128), ("dsgd_awc", 512)])
 @pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("topology,n,er_p,d", SHAPES + [("er_mh", 256, 0.05, 300_008), ("ring", 200, 0.0, 200_008)])
 def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, rule, threads):

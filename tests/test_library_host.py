@@ -23,6 +23,17 @@ def test_every_declared_symbol_is_exported():
         assert hasattr(lib, name), name
 
 
+def test_general_weight_tables_are_kept_bit_for_bit():
+    """A caller-supplied doubly-stochastic CSR weight matrix comes back from the builder unchanged, and is
+    doubly stochastic by the checks the paper's Assumption A.3 names (unit row and column sums, symmetry here)."""
+    rowptr, col, val, W = inputs.random_doubly_stochastic(40, 0.2, 77)
+    topo = B.topology_build(B.CSR_WEIGHTS, 40, rowptr, col, val)
+    r2, c2, v2 = topo.tables_host(0)
+    assert np.array_equal(r2, rowptr) and np.array_equal(c2, col) and np.array_equal(v2.view(np.uint32), val.view(np.uint32))
+    assert np.allclose(W.sum(0), 1.0, atol=1e-6) and np.allclose(W.sum(1), 1.0, atol=1e-6) and np.array_equal(W, W.T)
+    assert np.all(np.diag(W) > 0) and np.array_equal(_dense_from_csr(40, r2, c2, v2).astype(np.float64), W)
+
+
 def test_status_strings():
     lib = B.raw()
     assert lib.dlm_status_string(0) == b"ok"
