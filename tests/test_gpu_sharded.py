@@ -62,11 +62,12 @@ CASES = [  # (topology, n, d, gradient dtype, row padding of the per-rank buffer
     ("er_mh", 256, 8_200, "f32", 0),           # cfg5's graph
     ("bipartite_match", 12, 1_000, "f32", 0),  # time-varying, a different halo every slot
     ("complete", 6, 5, "f32", 3),              # fewer columns than a tile, every row needs every other
+    ("static_exp", 16, 10_003, "bf16", 5),     # bf16 gradients with a ragged last column group (row stride d + 5)
 ]
 
 
 @pytest.mark.parametrize("rule", ["decentlam", "dmsgd"])
-@pytest.mark.parametrize("ranks", [2, 4, 8])
+@pytest.mark.parametrize("ranks", [1, 2, 4, 8])
 @pytest.mark.parametrize("topology,n,d,g_dtype,pad", CASES)
 def test_sharded_calls_reproduce_the_unsharded_step_bitwise(rule, ranks, topology, n, d, g_dtype, pad):
     from paper_2104_11981_b200 import binding as B
