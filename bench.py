@@ -184,8 +184,19 @@ def aggregate_over_ranks(dist, seconds, units, device):
     return float(t.item()), float(u.item())
 
 
-def oracle_sample(workload, budget_s=20.0):
-    """Time the CPU oracle's DecentLaM step, as it stands, on a column slab of the workload."""
+def workload_config(args, w, n, d, world, g_esz):
+    """The `config` object of the JSON line: the same for both arms."""
+    return {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else "") +
+                        (f" (tuning {args.tuning})" if args.tuning else ""),
+            "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype, "beta": w.beta, "gamma": w.gamma,
+            "parallelism": "replicas only" if world > 1 else "1 gpu",
+            "l2": f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"}
+
+
+def oracle_sample(workload, budget_s=20.0, steps=None, warmup=0, wall_limit_s=150.0):
+    """Time the CPU oracle's DecentLaM step, as it stands, on a column slab of the workload.
+    steps=None: as many steps as fit budget_s (3 to 50), median step time.  steps=K: `warmup` untimed steps,
+    then exactly K timed ones; the slab is halved until K steps fit wall_limit_s."""
     import numpy as np
 
     import oracle
@@ -208,13 +219,28 @@ def oracle_sample(workload, budget_s=20.0):
     times = []
     t_begin = time.perf_counter()
     k = 0
-    while k < 3 or (time.perf_counter() - t_begin < budget_s and k < 50):
+    if steps is not None:
+        t0 = time.perf_counter()  # the first warm-up step doubles as the probe that sizes the slab
+        x, m = oracle.decentlam_step(Ws[0], x, m, g, np.float32(w.beta), np.float32(w.gamma), threads)
+        probe = time.perf_counter() - t0
+        k = 1
+        while steps * probe > wall_limit_s and cols > (1 << 12):
+            cols //= 2
+            probe /= 2
+            x, m, g = (np.ascontiguousarray(a[:, :cols]) for a in (x, m, g))
+        while k < max(1, warmup):
+            x, m = oracle.decentlam_step(Ws[k % period], x, m, g, np.float32(w.beta), np.float32(w.gamma), threads)
+            k += 1
+        budget_s = float("inf")
+    while (steps is not None and len(times) < steps) or \
+            (steps is None and (k < 3 or (time.perf_counter() - t_begin < budget_s and k < 50))):
         t0 = time.perf_counter()
         x, m = oracle.decentlam_step(Ws[k % period], x, m, g, np.float32(w.beta), np.float32(w.gamma), threads)
         times.append(time.perf_counter() - t0)
         k += 1
+    mean = sum(times) / len(times)
     times.sort()
-    med = times[len(times) // 2]
+    med = mean if steps is not None else times[len(times) // 2]  # K timed steps: total time / K
     single = []
     for k in range(2):                      # the same oracle on one thread, for the per-core figure
         t0 = time.perf_counter()
@@ -223,7 +249,8 @@ def oracle_sample(workload, budget_s=20.0):
     return {"value": w.n * cols / med, "unit": UNIT, "cores": threads, "kind": "oracle",
             "single_thread_value": w.n * cols / min(single),
             "sample": f"{workload}: {len(times)} DecentLaM steps of the double-precision dense-W oracle on a "
-                      f"[{w.n} x {cols}] column slab (median), {threads} threads"}, med, w.n * cols
+                      f"[{w.n} x {cols}] column slab ({'mean of the timed steps' if steps is not None else 'median'}), "
+                      f"{threads} threads"}, med, w.n * cols
 
 
 def oracle_lsq_sample(workload, A, b, iterations=3):
@@ -258,13 +285,15 @@ def run_reference(args):
     oracle_build.build()
     from paper_2104_11981_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
-    # each "step" is one oracle step on the bounded slab; warmup + steps of them
-    base, med, units = oracle_sample(args.workload, budget_s=min(60.0, 2.0 * (args.steps + args.warmup)))
+    # each "step" is one oracle step on the bounded slab: `warmup` untimed, then exactly `steps` timed
+    base, med, units = oracle_sample(args.workload, steps=args.steps, warmup=args.warmup)
+    d = args.columns if args.columns else w.d
     line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": med * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "n": w.n, "d": w.d, "topology": w.topology,
-                       "note": "CPU oracle on host cores; each step is a bounded column slab"},
+            "config": workload_config(args, w, w.n, d, int(os.environ.get("WORLD_SIZE", "1")),
+                                      2 if w.g_dtype == "bf16" else 4),
+            "note": "the CPU oracle on the host cores; each step is one oracle step on a bounded column slab",
             "cpu_baseline": base,
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -517,10 +546,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": job_secs / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload + (f" (columns overridden to {d})" if args.columns else "") +
-                                   (f" (tuning {args.tuning})" if args.tuning else ""), "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype,
-                       "beta": w.beta, "gamma": w.gamma, "parallelism": "replicas only" if world > 1 else "1 gpu",
-                       "l2": f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"},
+            "config": workload_config(args, w, n, d, world, g_esz),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic_total, "traffic_detail": traffic_detail, "peak_kind": f"of {peak_kind}",
                          "kernel": "step_tma_kernel<decentlam>", "algorithmic_bytes_per_launch": bytes_per_np * n * d,

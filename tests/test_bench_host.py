@@ -55,6 +55,15 @@ def test_reference_arm_prints_one_line_on_rank0_only():
     assert rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["cores"] >= 1
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["e2e"]["value"] == rec["value"]
     assert rec["config"]["workload"] == "cfg2" and rec["higher_is_better"] is True
+    # the config object is the one the GPU arm prints for the same arguments, and exactly `steps` steps were timed
+    import argparse
+
+    import bench
+    from paper_2104_11981_b200 import inputs
+    w = inputs.WORKLOADS["cfg2"]
+    ours = bench.workload_config(argparse.Namespace(workload="cfg2", columns=0, tuning=""), w, w.n, w.d, 2, 4)
+    assert rec["config"] == ours
+    assert rec["steps"] == 1 and rec["cpu_baseline"]["sample"].startswith("cfg2: 1 DecentLaM steps")
     env["RANK"] = "1"
     r1 = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                          "--steps", "1", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=300)
