@@ -413,6 +413,9 @@ DLM_API int dlm_kernel_error(int* flag);
  *           (negative = automatic: 0.55 of the L2 size when H is between that and twice the L2
  *           size, else none)
  *   knob 12 block size of the compact-table merged kernel (128, 256 or 512)
+ *   knob 13 1 = the compact-table merged kernel never uses its 256-bit global loads and stores (the
+ *           automatic choice uses them on more than 128 nodes when x, m and their rows are aligned to
+ *           32 bytes and d is a multiple of 8)
  * Results do not depend on the knobs, with one exception: the merged-staging kernels (knob 7 = 2 or 3,
  * the default on long rows: 8 or more entries; 12 or more for dsgd_step above 128 nodes) arrange the same
  * sum differently and agree with the other paths, and with each other, to rounding, not bitwise.

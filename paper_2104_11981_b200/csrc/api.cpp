@@ -276,7 +276,8 @@ int dlm_set_tuning(int knob, int value) {
     case 9: g_lsq_tune_bulk = value; return DLM_OK;
     case 10: g_pmsgd_tune_cap = value; return DLM_OK;
     case 11: g_l2_keep_permille = value; return DLM_OK;
-    case 12: return dlm_compact_set_tuning(knob, value);
+    case 12:
+    case 13: return dlm_compact_set_tuning(knob, value);
     default: return DLM_ERR_KIND;
     }
 }

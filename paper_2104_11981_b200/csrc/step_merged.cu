@@ -47,11 +47,30 @@ __device__ __forceinline__ float4 lds128(uint32_t addr) {
     return v;
 }
 
+// 256-bit global accesses (32-byte aligned addresses): a lane's eight consecutive columns in one request
+__device__ __forceinline__ void ldg256(const float* p, Pack<4>& lo, Pack<4>& hi) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(lo.v[0]), "=f"(lo.v[1]), "=f"(lo.v[2]), "=f"(lo.v[3]), "=f"(hi.v[0]), "=f"(hi.v[1]),
+                   "=f"(hi.v[2]), "=f"(hi.v[3])
+                 : "l"(p)
+                 : "memory");
+}
+__device__ __forceinline__ void stg256(float* p, const Pack<4>& lo, const Pack<4>& hi) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "f"(lo.v[0]), "f"(lo.v[1]),
+                 "f"(lo.v[2]), "f"(lo.v[3]), "f"(hi.v[0]), "f"(hi.v[1]), "f"(hi.v[2]), "f"(hi.v[3])
+                 : "memory");
+}
+__device__ __forceinline__ Pack<4> pick(bool second, const Pack<4>& a, const Pack<4>& b) {
+    return {{second ? b.v[0] : a.v[0], second ? b.v[1] : a.v[1], second ? b.v[2] : a.v[2], second ? b.v[3] : a.v[3]}};
+}
+
 struct MergedGeom {
     int C;          // tile columns (power of two, 32 .. 256)
     int cv_shift;   // log2(C / 4)
     int tables_in_smem;
     int prefetch_m;        // DecentLaM: request the tile's m lines into L2 before waiting for the tile
+    int wide;              // compact kernel, 32-column tiles: a lane's two column groups are adjacent and its
+                           // global loads and stores are single 256-bit requests (whole 128-byte lines per row)
     uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
     uint32_t v_off, g_off; // byte offsets of the staged-value tile and of the g landing area inside the stage
     uint32_t stage_bytes;
@@ -291,6 +310,7 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     geo.cv_shift = ilog2(C / 4);
     // measured: +3 to +8 % with tiles of 64 columns or more (up to 128 nodes); with 256 nodes and
     // 32-column tiles the extra requests cost 6 % instead
+    geo.wide = 0;
     geo.prefetch_m = C >= 64;
     geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
     geo.num_tiles = (a.d + C - 1) / C;
@@ -325,8 +345,12 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
 // off-diagonal entries (Metropolis-Hastings and all built-in graphs: a few dozen weights).
 // Blob layout (a.compact): rowrec u32[n] {i | len << 8 | first << 16} in processing order, S f32[n],
 // wself f32[n], wlut f32[nw + 1] (last = 0, the filler's weight), cent u16[noff] {col | widx << 8}.
+// WIDE (32-column tiles: four lanes per row): a lane's two column groups are adjacent, and its m load and
+// its x, m stores are single 256-bit requests, so that the four lanes of a row touch one whole 128-byte
+// line per request instead of half a line in each of two; needs rows and bases aligned to 32 bytes and
+// d a multiple of 8.  Same sums, same results.
 // ---------------------------------------------------------------------------------------------
-template <int RULE, typename GT, int THREADS, int MIN_CTAS>
+template <int RULE, typename GT, int THREADS, int MIN_CTAS, bool WIDE>
 __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                                          const __grid_constant__ CUtensorMap tm_g,
                                                                          dlm_step_args a, MergedGeom geo) {
@@ -378,6 +402,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
     const int glane = (threadIdx.x & 31) & (L - 1);
     const int row_shift = geo.cv_shift + 4;  // log2 of the row pitch in bytes (C * 4)
     const uint32_t filler_w = (uint32_t)a.compact_nw << 8;
+    constexpr bool wide = WIDE;
 
     // DmSGD: pass-1 items per thread whose m is fetched before the wait for the tile (all of them at 256 and
     // at 512 threads for tiles of 8192 elements)
@@ -460,14 +485,26 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
             // column groups {q, q + L}; with four lanes per row, neighbouring rows take the two halves in
             // opposite order so that a quarter warp still covers all 32 banks
             const int par = (L == 4) ? (slot & 1) : 0;
-            const int off0 = (L == 4 ? glane + 4 * par : glane) * 4;
-            const int off1 = (L == 4 ? glane + 4 * (1 - par) : glane + L) * 4;
+            // wide: the lane owns the columns [8 glane, 8 glane + 8); which half it loads first alternates with the
+            // row, so that a quarter warp still covers all 32 banks
+            const int off0 = wide ? (2 * glane + par) * 4 : (L == 4 ? glane + 4 * par : glane) * 4;
+            const int off1 = wide ? (2 * glane + 1 - par) * 4 : (L == 4 ? glane + 4 * (1 - par) : glane + L) * 4;
             const long long c0 = tile_base + off0, c1 = tile_base + off1;
-            const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;
+            const bool st0 = live && c0 < a.d, st1 = live && c1 < a.d;  // wide: d is a multiple of 8, st0 == st1
+            const size_t wide_at = (size_t)i * a.ld + tile_base + 8 * glane;
             Pack<4> m0 = {{0.f, 0.f, 0.f, 0.f}}, m1 = {{0.f, 0.f, 0.f, 0.f}};
-            if (LAM) {
-                if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);  // in flight during the loop
-                if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+            if (LAM) {  // in flight during the loop
+                if (wide) {
+                    if (st0) {
+                        Pack<4> lo, hi;
+                        ldg256(a.m + wide_at, lo, hi);
+                        m0 = pick(par != 0, lo, hi);
+                        m1 = pick(par != 0, hi, lo);
+                    }
+                } else {
+                    if (st0) m0 = ld_f32<4>(a.m + (size_t)i * a.ld + c0);
+                    if (st1) m1 = ld_f32<4>(a.m + (size_t)i * a.ld + c1);
+                }
             }
             float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t vb0 = smem_u32(vs) + off0 * 4, vb1 = smem_u32(vs) + off1 * 4;
@@ -490,14 +527,15 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
             // self weight: the stored diagonal for DecentLaM's v-sum, the exact remainder for the averages
             const float S_i = LAM ? Ssum[slot] : 0.f;
             const float w_ii = LAM ? wself[slot] : (live ? __int_as_float(a.selfw[slot]) : 0.f);
+            Pack<4> xn2[2], mn2[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int off = h ? off1 : off0;
                 const Pack<4> vi = ld_f32<4>(vs + i * C + off);
-                Pack<4> xn;
+                Pack<4>& xn = xn2[h];
                 if (LAM) {
                     const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
-                    Pack<4> mn;
+                    Pack<4>& mn = mn2[h];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const float mix = fmaf(w_ii, vi.v[u], h ? acc1[u] : acc0[u]);  // self term of the v-sum
@@ -505,7 +543,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
                         mn.v[u] = fmaf(a.beta, h ? m1.v[u] : m0.v[u], gt);
                         xn.v[u] = fmaf(-a.gamma, mn.v[u], xi.v[u]);
                     }
-                    if (h ? st1 : st0) st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
+                    if (!wide && (h ? st1 : st0)) st_f32<4>(a.m + (size_t)i * a.ld + (h ? c1 : c0), mn);
                 } else {
 #pragma unroll
                     for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(w_ii, vi.v[u], h ? acc1[u] : acc0[u]);
@@ -515,7 +553,11 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
                         for (int u = 0; u < 4; ++u) xn.v[u] = fmaf(-a.gamma, gi.v[u], xn.v[u]);
                     }
                 }
-                if (h ? st1 : st0) st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
+                if (!wide && (h ? st1 : st0)) st_f32<4>(a.x + (size_t)i * a.ld + (h ? c1 : c0), xn);
+            }
+            if (wide && st0) {  // the lower columns are the first group's on even rows, the second group's on odd rows
+                if (LAM) stg256(a.m + wide_at, pick(par != 0, mn2[0], mn2[1]), pick(par != 0, mn2[1], mn2[0]));
+                stg256(a.x + wide_at, pick(par != 0, xn2[0], xn2[1]), pick(par != 0, xn2[1], xn2[0]));
             }
         }
         if (it + 1 < my_tiles) {
@@ -526,6 +568,7 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
     }
 }
 
+int g_tune_compact_wide = 0;     // knob 13: 1 = never use the 256-bit global requests
 int g_tune_compact_threads = 0;  // knob 12: block size of the compact-table kernel (128, 256 or 512), 0 = auto
 
 // Compact-table merged kernel.  DLM_ERR_UNSUPPORTED if the slot has no compact tables or the shape does
@@ -564,6 +607,10 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     geo.C = C;
     geo.cv_shift = ilog2(C / 4);
     geo.prefetch_m = C >= 64;
+    // 32-column tiles give a row four lanes: with two separate 16-byte groups per lane every global request
+    // touches half a 128-byte line per row; with adjacent groups and 256-bit requests it touches whole lines
+    geo.wide = C == 32 && a.ld % 8 == 0 && a.d % 8 == 0 && (uintptr_t)a.x % 32 == 0 && (uintptr_t)a.m % 32 == 0 &&
+               g_tune_compact_wide != 1;
     geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
     geo.num_tiles = (a.d + C - 1) / C;
     CUtensorMap tm_x, tm_g;
@@ -578,15 +625,23 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     //     before the wait for the tile (256 threads: 10 to 15 % slower, 128: 40 %).
     //   DSGD (no momentum, the lightest pass 2): 256 threads, three CTAs per SM.
     //   Up to 16 nodes (tiles of 256 columns, a warp per row): 128 threads for every rule.
+    //   With 256-bit global requests (32-column tiles, i.e. more than 128 nodes, rows and bases aligned to 32 bytes):
+    //     DecentLaM 256 threads (5 to 7 % ahead of the best block size without them on rings, exponential and
+    //     Erdos-Renyi graphs of 200 and 256 nodes; 128 threads lose 10 %), 512 with bf16 gradients; DmSGD 512 on
+    //     short rows, 256 from about 14 entries per row on and with bf16 gradients; DSGD 256.
     int threads = g_tune_compact_threads;
     if (threads != 128 && threads != 256 && threads != 512) {
         if (a.n <= 16) threads = 128;
-        else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;
+        else if (geo.wide) {
+            if (LAM) threads = bf16 ? 512 : 256;
+            else if (RULE == DLM_RULE_DMSGD) threads = (bf16 || (long long)a.nnz > 14LL * a.n) ? 256 : 512;
+            else threads = 256;
+        } else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;
         else threads = RULE == DLM_RULE_DMSGD ? 512 : 256;
     }
 #define DLM_COMPACT_LAUNCH(T, M)                                                                               \
     {                                                                                                          \
-        auto kern = step_compact_kernel<RULE, GT, T, M>;                                                             \
+        auto kern = geo.wide ? step_compact_kernel<RULE, GT, T, M, true> : step_compact_kernel<RULE, GT, T, M, false>; \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
             return DLM_ERR_CUDA;                                                                               \
         kern<<<(unsigned)grid, T, smem, stream>>>(tm_x, tm_g, a, geo);                                         \
@@ -602,8 +657,8 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
 }  // namespace
 
 int dlm_compact_set_tuning(int knob, int value) {
-    (void)knob;
-    g_tune_compact_threads = value;
+    if (knob == 13) g_tune_compact_wide = value;
+    else g_tune_compact_threads = value;
     return DLM_OK;
 }
 

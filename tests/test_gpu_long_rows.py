@@ -42,12 +42,61 @@ def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, rule, threa
     from paper_2104_11981_b200 import binding as B
     try:
         B.set_tuning(7, 3); B.set_tuning(12, threads)
-        _run(topology, n, er_p, d, rule, g_dtype)
+        _run(topology, n, er_p, d, rule, g_dtype)   # above 128 nodes: with the 256-bit global requests
+        if n > 128:
+            B.set_tuning(13, 1)                     # ... and without them
+            _run(topology, n, er_p, d, rule, g_dtype)
+            B.set_tuning(13, 0)
         if threads == 512:
             B.set_tuning(7, 2)
             _run(topology, n, er_p, d, rule, g_dtype)
     finally:
-        B.set_tuning(7, 0); B.set_tuning(12, 0)
+        B.set_tuning(7, 0); B.set_tuning(12, 0); B.set_tuning(13, 0)
+
+
+@pytest.mark.parametrize("rule", ["decentlam", "dmsgd", "dsgd_atc", "dsgd_awc"])
+@pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
+def test_wide_global_requests_change_nothing(rule, g_dtype):
+    """Above 128 nodes the compact-table kernel moves m and x with 256-bit requests when rows and bases are
+    aligned to 32 bytes and d is a multiple of 8.  Bitwise the results without them, over the whole state,
+    at every block size; a column count of 4 mod 8 and a base that is only 16-byte aligned take the
+    128-bit path by themselves (and must still agree with the plain mixing loop to rounding)."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    n, beta, gamma = 200, 0.9, 0.05
+    topo, _ = build_both("er_mh", n, graph_seed=SEED + 3, er_p=0.06)
+    gt = torch.bfloat16 if g_dtype == "bf16" else torch.float32
+    try:
+        for d, shift in ((40_008, 0), (40_004, 0), (40_008, 4)):
+            ld = d + shift + (8 - (d + shift) % 8) % 8 + 8
+            buf = {k: inputs.normal_torch((n, ld), s, SEED + i, dev) for i, (k, s) in
+                   enumerate((("x", 0.02), ("m", 1e-3), ("g", 1e-3)))}
+            x0, m0 = buf["x"][:, shift:shift + d], buf["m"][:, shift:shift + d]
+            g = buf["g"].to(gt)[:, :d]                           # 16-byte aligned for either gradient type
+            results = {}
+            for wide_off in (0, 1):
+                for threads in (128, 256, 512):
+                    B.set_tuning(7, 3); B.set_tuning(12, threads); B.set_tuning(13, wide_off)
+                    xb, mb = buf["x"].clone(), buf["m"].clone()
+                    x, m = xb[:, shift:shift + d], mb[:, shift:shift + d]
+                    for k in range(3):
+                        lib_rule(rule, topo, k, x, m, g, beta, gamma)
+                    torch.cuda.synchronize()
+                    assert B.kernel_error() == 0
+                    results[(wide_off, threads)] = (xb, mb)     # whole buffers: the padding must stay untouched
+            ref = results[(1, 128)]
+            for key, (xb, mb) in results.items():
+                assert torch.equal(xb, ref[0]) and torch.equal(mb, ref[1]), (d, shift, key)
+            B.set_tuning(7, 1)                                   # the plain mixing loop
+            xb, mb = buf["x"].clone(), buf["m"].clone()
+            x, m = xb[:, shift:shift + d], mb[:, shift:shift + d]
+            for k in range(3):
+                lib_rule(rule, topo, k, x, m, g, beta, gamma)
+            assert rel_l2(to64(xb), to64(ref[0])) <= 1e-6
+            if rule in ("decentlam", "dmsgd"):
+                assert rel_l2(to64(mb), to64(ref[1])) <= 1e-6
+    finally:
+        B.set_tuning(7, 0); B.set_tuning(12, 0); B.set_tuning(13, 0)
 
 
 def _run(topology, n, er_p, d, rule, g_dtype):
