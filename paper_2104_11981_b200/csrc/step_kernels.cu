@@ -446,8 +446,15 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     //              entries per row on below that
     //   DSGD       from 32 nodes on (rings, one-peer, mesh: +3 to +15 %); from 12 nodes on for
     //              adapt-then-combine (+3 to +15 %) and, with three or more entries per row, for adapt-with-combine
+    //   DecentLaM with bf16 gradients (they land inside the tile of staged values there, so a third CTA fits per
+    //              SM): from 5 entries per row on at 32 nodes or more (exponential graphs of 32 / 64 nodes, the
+    //              symmetric exponential graph and the mesh of 64: +4 to +10 % sustained; rings, one-peer graphs
+    //              and 16 nodes: behind); the plain loop up to 8 nodes (complete graph of 8: compact -11 %)
     if (a.compact) {
-        if (RULE == DLM_RULE_DECENTLAM) want_merged = a.max_degree >= 8;
+        if (RULE == DLM_RULE_DECENTLAM) {
+            want_merged = a.max_degree >= 8;
+            if (sizeof(GT) == 2) want_merged = a.n > 8 && (a.max_degree >= 8 || (a.n >= 32 && a.max_degree >= 5));
+        }
         if (RULE == DLM_RULE_DMSGD) want_merged = a.n >= 64 || a.max_degree >= 6;
         if (RULE == DLM_RULE_DSGD_ATC) want_merged = a.n >= 12;
         if (RULE == DLM_RULE_DSGD_AWC) want_merged = a.n >= 32 || (a.n >= 12 && a.max_degree >= 3);

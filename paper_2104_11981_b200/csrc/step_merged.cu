@@ -69,6 +69,7 @@ struct MergedGeom {
     int cv_shift;   // log2(C / 4)
     int tables_in_smem;
     int prefetch_m;        // DecentLaM: request the tile's m lines into L2 before waiting for the tile
+    int g_in_v;            // compact kernel, DecentLaM with bf16 gradients: g lands in the last quarter of the v tile
     int wide;              // compact kernel, 32-column tiles: a lane's two column groups are adjacent and its
                            // global loads and stores are single 256-bit requests (whole 128-byte lines per row)
     uint32_t x_bytes;      // fp32 tile bytes (128-byte multiple)
@@ -310,6 +311,7 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
     geo.cv_shift = ilog2(C / 4);
     // measured: +3 to +8 % with tiles of 64 columns or more (up to 128 nodes); with 256 nodes and
     // 32-column tiles the extra requests cost 6 % instead
+    geo.g_in_v = 0;
     geo.wide = 0;
     geo.prefetch_m = C >= 64;
     geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
@@ -345,6 +347,10 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
 // off-diagonal entries (Metropolis-Hastings and all built-in graphs: a few dozen weights).
 // Blob layout (a.compact): rowrec u32[n] {i | len << 8 | first << 16} in processing order, S f32[n],
 // wself f32[n], wlut f32[nw + 1] (last = 0, the filler's weight), cent u16[noff] {col | widx << 8}.
+// DecentLaM with bf16 gradients: the gradients' landing area is the last quarter of the tile that pass 1
+// fills with v (every thread takes its items' gradients into registers, a barrier, then v is written
+// over them), so that x and v are all a CTA stages, as with fp32 gradients: 64 KB per 8192 node-columns,
+// three CTAs per SM instead of two.  Needs n C <= 8192 (a thread's share must fit its registers).
 // WIDE (32-column tiles: four lanes per row): a lane's two column groups are adjacent, and its m load and
 // its x, m stores are single 256-bit requests, so that the four lanes of a row touch one whole 128-byte
 // line per request instead of half a line in each of two; needs rows and bases aligned to 32 bytes and
@@ -437,7 +443,35 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
         }
         // pass 1.  DecentLaM: v = g - (x - r) / gamma, r = row 0's value of the column.  DmSGD: m' = beta m + g,
         // y = x - gamma m'.  Adapt-then-combine: y = x - gamma g.  Adapt-with-combine averages x as it is.
-        if (RULE != DLM_RULE_DSGD_AWC) {
+        if (LAM && sizeof(GT) == 2 && geo.g_in_v) {
+            // bf16 gradients landed inside the tile that v is about to fill (its last quarter): every thread
+            // first takes all of its gradients into registers, then, after a barrier, writes v over them.
+            // An item's four gradients sit at element 4 e of the dense [n][C] landing area.
+            constexpr int kOwn = (2048 + THREADS - 1) / THREADS;  // items per thread: n C <= 8192
+            uint2 graw[kOwn];
+#pragma unroll
+            for (int k = 0; k < kOwn; ++k) {
+                const int e = threadIdx.x + k * THREADS;
+                graw[k] = make_uint2(0u, 0u);
+                if (e < items) graw[k] = *reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(gs) + 4 * e);
+            }
+            __syncthreads();
+#pragma unroll
+            for (int k = 0; k < kOwn; ++k) {
+                const int e = threadIdx.x + k * THREADS;
+                if (e < items) {
+                    const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
+                    const Pack<4> xi = ld_f32<4>(xs + i * C + off), ref = ld_f32<4>(xs + off);
+                    const float gi[4] = {__uint_as_float(graw[k].x << 16), __uint_as_float(graw[k].x & 0xffff0000u),
+                                         __uint_as_float(graw[k].y << 16), __uint_as_float(graw[k].y & 0xffff0000u)};
+                    Pack<4> v;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v.v[u] = fmaf(-a.inv_gamma, xi.v[u] - ref.v[u], gi[u]);
+                    st_f32<4>(vs + i * C + off, v);
+                }
+            }
+            __syncthreads();
+        } else if (RULE != DLM_RULE_DSGD_AWC) {
             int k = 0;
             for (int e = threadIdx.x; e < items; e += THREADS, ++k) {
                 const int i = e >> geo.cv_shift, off = (e & cv_mask) * 4;
@@ -591,10 +625,12 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
         const size_t xb = ((size_t)a.n * C * 4 + 127) & ~(size_t)127;
         const size_t gb = ((size_t)a.n * C * sizeof(GT) + 127) & ~(size_t)127;
         geo.x_bytes = (uint32_t)xb;
-        if (LAM) {  // [x | v | g]: for fp32 gradients v overwrites g in place
+        // bf16 gradients can land inside the v tile when a thread can hold all of its items' gradients
+        geo.g_in_v = LAM && bf16 && (size_t)a.n * C <= 8192;
+        if (LAM) {  // [x | v | g]: for fp32 gradients v overwrites g in place, bf16 gradients land in v's last quarter
             geo.v_off = (uint32_t)xb;
-            geo.g_off = (uint32_t)(bf16 ? 2 * xb : xb);
-            geo.stage_bytes = (uint32_t)(bf16 ? 2 * xb + gb : 2 * xb);
+            geo.g_off = (uint32_t)(!bf16 ? xb : geo.g_in_v ? 2 * xb - gb : 2 * xb);
+            geo.stage_bytes = (uint32_t)(bf16 && !geo.g_in_v ? 2 * xb + gb : 2 * xb);
         } else {    // [x (becomes y) | g]
             geo.v_off = 0;
             geo.g_off = (uint32_t)xb;
@@ -627,13 +663,13 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
     //   Up to 16 nodes (tiles of 256 columns, a warp per row): 128 threads for every rule.
     //   With 256-bit global requests (32-column tiles, i.e. more than 128 nodes, rows and bases aligned to 32 bytes):
     //     DecentLaM 256 threads (5 to 7 % ahead of the best block size without them on rings, exponential and
-    //     Erdos-Renyi graphs of 200 and 256 nodes; 128 threads lose 10 %), 512 with bf16 gradients; DmSGD 512 on
+    //     Erdos-Renyi graphs of 200 and 256 nodes; 128 threads lose 10 %; 512 lose 8 % with bf16 gradients); DmSGD 512 on
     //     short rows, 256 from about 14 entries per row on and with bf16 gradients; DSGD 256.
     int threads = g_tune_compact_threads;
     if (threads != 128 && threads != 256 && threads != 512) {
         if (a.n <= 16) threads = 128;
         else if (geo.wide) {
-            if (LAM) threads = bf16 ? 512 : 256;
+            if (LAM) threads = 256;
             else if (RULE == DLM_RULE_DMSGD) threads = (bf16 || (long long)a.nnz > 14LL * a.n) ? 256 : 512;
             else threads = 256;
         } else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;

@@ -54,6 +54,41 @@ def test_compact_table_kernel_sampled(topology, n, er_p, d, g_dtype, rule, threa
         B.set_tuning(7, 0); B.set_tuning(12, 0); B.set_tuning(13, 0)
 
 
+@pytest.mark.parametrize("topology,n,er_p", [("static_exp", 64, 0.0), ("er_mh", 200, 0.06), ("mesh", 36, 0.0)])
+def test_bf16_gradients_landing_inside_the_value_tile(topology, n, er_p):
+    """DecentLaM with bf16 gradients: the compact-table kernel lands g in the last quarter of the tile that
+    pass 1 fills with v.  With tiles of 256 columns (knob 1) a thread's share no longer fits its registers and
+    g keeps a landing area of its own: same arithmetic, bitwise the same state; both within 1e-6 of the
+    plain mixing loop, which is what these graphs took before."""
+    from paper_2104_11981_b200 import binding as B
+    dev = torch.device("cuda:0")
+    d, beta, gamma = 150_008, 0.9, 0.05
+    topo, _ = build_both(topology, n, graph_seed=SEED + 5, er_p=er_p or 0.05)
+    x0 = (inputs.normal_torch((1, d), 0.02, SEED + 21, dev) + inputs.normal_torch((n, d), 1e-3, SEED + 22, dev)).contiguous()
+    m0 = inputs.normal_torch((n, d), 1e-3, SEED + 23, dev)
+    g = inputs.normal_torch((n, d), 1e-3, SEED + 24, dev).to(torch.bfloat16)
+    out = {}
+    try:
+        for name, knobs in (("inside", {7: 3}), ("own area", {7: 3, 1: 256}), ("plain", {7: 1})):
+            if name == "own area" and n > 128:
+                continue                            # 256-column tiles of more than 128 rows do not fit an SM
+            for k, v in knobs.items():
+                B.set_tuning(k, v)
+            x, m = x0.clone(), m0.clone()
+            for k in range(4):
+                B.decentlam_step(topo, k, x, m, g, beta, gamma)
+            torch.cuda.synchronize()
+            assert B.kernel_error() == 0
+            out[name] = (x, m)
+            B.set_tuning(7, 0); B.set_tuning(1, 0)
+        if "own area" in out:
+            assert torch.equal(out["inside"][0], out["own area"][0]) and torch.equal(out["inside"][1], out["own area"][1])
+        assert rel_l2(to64(out["inside"][0]), to64(out["plain"][0])) <= 1e-6
+        assert rel_l2(to64(out["inside"][1]), to64(out["plain"][1])) <= 1e-6
+    finally:
+        B.set_tuning(7, 0); B.set_tuning(1, 0)
+
+
 @pytest.mark.parametrize("rule", ["decentlam", "dmsgd", "dsgd_atc", "dsgd_awc"])
 @pytest.mark.parametrize("g_dtype", ["f32", "bf16"])
 def test_wide_global_requests_change_nothing(rule, g_dtype):
