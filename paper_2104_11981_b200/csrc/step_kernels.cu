@@ -446,14 +446,18 @@ int launch_tma(const dlm_step_args& a, cudaStream_t stream) {
     //              entries per row on below that
     //   DSGD       from 32 nodes on (rings, one-peer, mesh: +3 to +15 %); from 12 nodes on for
     //              adapt-then-combine (+3 to +15 %) and, with three or more entries per row, for adapt-with-combine
-    //   DecentLaM with bf16 gradients (they land inside the tile of staged values there, so a third CTA fits per
-    //              SM): from 5 entries per row on at 32 nodes or more (exponential graphs of 32 / 64 nodes, the
-    //              symmetric exponential graph and the mesh of 64: +4 to +10 % sustained; rings, one-peer graphs
-    //              and 16 nodes: behind); the plain loop up to 8 nodes (complete graph of 8: compact -11 %)
+    //   Over runs of a hundred steps and more the SM clock settles near 1.65 GHz under the power cap, and there
+    //   DecentLaM gains from the merged pass much earlier than in short bursts (748 M node-parameters, 150 steps):
+    //   from 5 entries per row on at 12 nodes or more with fp32 gradients (exponential graphs of 12 / 20 / 24 / 32 /
+    //   48 / 64 nodes +7 / +14 / +8 / +7 / +12 / +8 %, meshes of 25 / 36 / 100 nodes +6 / +10 / +9 %; level at 16 nodes and on
+    //   the mesh of 64; rings and one-peer graphs 0 to 3 % behind, so they keep the plain loop), and at 20 nodes or
+    //   more with bf16 gradients (exponential graphs of 20 / 24 / 32 / 48 / 64 nodes +18 / +13 / +10 / +16 / +10 %, meshes of
+    //   25 / 36 / 64 +10 / +12 / +4 %, symmetric exponential graphs +7 to +10 %; 16 nodes 3 % behind, the complete graph
+    //   of 8 nodes 11 % behind, the mesh of 100 nodes 2 % behind).
     if (a.compact) {
         if (RULE == DLM_RULE_DECENTLAM) {
-            want_merged = a.max_degree >= 8;
-            if (sizeof(GT) == 2) want_merged = a.n > 8 && (a.max_degree >= 8 || (a.n >= 32 && a.max_degree >= 5));
+            if (sizeof(GT) == 2) want_merged = a.n > 8 && (a.max_degree >= 8 || (a.n >= 20 && a.max_degree >= 5));
+            else want_merged = a.max_degree >= 8 || (a.n >= 12 && a.max_degree >= 5);
         }
         if (RULE == DLM_RULE_DMSGD) want_merged = a.n >= 64 || a.max_degree >= 6;
         if (RULE == DLM_RULE_DSGD_ATC) want_merged = a.n >= 12;

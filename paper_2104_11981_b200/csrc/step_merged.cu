@@ -672,7 +672,12 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
             if (LAM) threads = 256;
             else if (RULE == DLM_RULE_DMSGD) threads = (bf16 || (long long)a.nnz > 14LL * a.n) ? 256 : 512;
             else threads = 256;
-        } else if (LAM) threads = (!bf16 && a.n >= 128) ? 128 : 256;
+        } else if (LAM) {
+            // fp32 gradients: 128 threads from 128 nodes on, and wherever five CTAs fit an SM's shared memory (small
+            // tiles: 20, 36, 100 nodes +5 / +5 / +2 %; four fit with 108 registers, against three of 256 threads)
+            const bool small_tiles = 5 * (smem + 1024) <= sm_total;
+            threads = (!bf16 && (a.n >= 128 || small_tiles)) ? 128 : 256;
+        }
         else threads = RULE == DLM_RULE_DMSGD ? 512 : 256;
     }
 #define DLM_COMPACT_LAUNCH(T, M)                                                                               \
