@@ -396,7 +396,7 @@ def side_workload(name, B, inputs, torch, dev, stream, peak, steps=20, repeats=5
     return {"n": w.n, "d": w.d, "topology": w.topology, "g_dtype": w.g_dtype, "steps_each": steps, "repeats": repeats,
             "ms_per_step": med, "ms_per_step_min": per_step[0], "value": w.n * w.d / (med * 1e-3), "unit": UNIT,
             "gbs": bytes_alg / (med * 1e-3) / 1e9, "frac": bytes_alg / (med * 1e-3) / 1e9 / peak,
-            "algorithmic_bytes_per_launch": bytes_alg, "clocks": clocks}
+            "algorithmic_bytes_per_launch": bytes_alg, "kernel": DOMINANT_KERNEL.get(name), "clocks": clocks}
 
 
 def run_ours(args):
