@@ -359,6 +359,7 @@ int launch_merged(const dlm_step_args& a, cudaStream_t stream) {
 template <int RULE, typename GT, int THREADS, int MIN_CTAS, bool WIDE>
 __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const __grid_constant__ CUtensorMap tm_x,
                                                                          const __grid_constant__ CUtensorMap tm_g,
+                                                                         const __grid_constant__ CUtensorMap tm_m,
                                                                          dlm_step_args a, MergedGeom geo) {
     constexpr bool LAM = RULE == DLM_RULE_DECENTLAM;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -376,6 +377,11 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
         mbar_expect_tx(bar, geo.tx_bytes);
         tma_load_2d(smem_u32(st), &tm_x, c0, 0, bar);
         tma_load_2d(smem_u32(st + geo.g_off), &tm_g, c0, 0, bar);
+        // DecentLaM reads m in pass 2 with plain loads, one per item just before its mixing loop: too short a loop
+        // to cover a trip to DRAM on tiles of 64 columns or more.  One bulk prefetch brings the tile's m box into
+        // L2 while the tile itself is on its way (no shared memory, no registers, no barrier: a hint).
+        if (LAM && geo.prefetch_m)
+            asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&tm_m), "r"(c0), "r"(0) : "memory");
     };
     if (threadIdx.x == 0) {
         mbar_init(bar, 1);
@@ -423,14 +429,6 @@ __global__ void __launch_bounds__(THREADS, MIN_CTAS) step_compact_kernel(const _
                 const long long c = tile_base + (e & cv_mask) * 4;
                 mpre[k] = {{0.f, 0.f, 0.f, 0.f}};
                 if (e < items && c < a.d) mpre[k] = ld_f32<4>(a.m + (size_t)(e >> geo.cv_shift) * a.ld + c);
-            }
-        }
-        if (LAM && geo.prefetch_m) {
-            const int seg_shift = geo.cv_shift - 3, segs = a.n << seg_shift;  // C / 32 segments per row
-            for (int e = threadIdx.x; e < 2 * segs; e += THREADS) {
-                const int sg = e >> 1;
-                const long long c = tile_base + (long long)(sg & ((1 << seg_shift) - 1)) * 32 + (e & 1) * 28;
-                if (c < a.d) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.m + (size_t)(sg >> seg_shift) * a.ld + c));
             }
         }
         if (!cta_wait(bar, (uint32_t)(it & 1))) {  // uniform decision: give up together
@@ -649,9 +647,11 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
                g_tune_compact_wide != 1;
     geo.tx_bytes = (uint32_t)((size_t)a.n * C * (4 + sizeof(GT)));
     geo.num_tiles = (a.d + C - 1) / C;
-    CUtensorMap tm_x, tm_g;
+    CUtensorMap tm_x, tm_g, tm_m;
     if (!make_map(&tm_x, a.x, false, a.n, a.d, a.ld, C) || !make_map(&tm_g, a.g, bf16, a.n, a.d, a.ldg, C))
         return DLM_ERR_UNSUPPORTED;
+    tm_m = tm_x;
+    if (LAM && !make_map(&tm_m, a.m, false, a.n, a.d, a.ld, C)) return DLM_ERR_UNSUPPORTED;
     const int tiles_per_cta = g_tune_tiles_per_cta > 0 ? g_tune_tiles_per_cta : 4;
     const long long grid = (geo.num_tiles + tiles_per_cta - 1) / tiles_per_cta;
     // Block size, measured on ring, exponential, Erdos-Renyi and complete graphs of 8 .. 256 nodes.
@@ -685,7 +685,7 @@ int launch_compact(const dlm_step_args& a, cudaStream_t stream) {
         auto kern = geo.wide ? step_compact_kernel<RULE, GT, T, M, true> : step_compact_kernel<RULE, GT, T, M, false>; \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) \
             return DLM_ERR_CUDA;                                                                               \
-        kern<<<(unsigned)grid, T, smem, stream>>>(tm_x, tm_g, a, geo);                                         \
+        kern<<<(unsigned)grid, T, smem, stream>>>(tm_x, tm_g, tm_m, a, geo);                                   \
     }
     if (threads == 128) DLM_COMPACT_LAUNCH(128, 3)
     else if (threads == 256) DLM_COMPACT_LAUNCH(256, 3)
