@@ -418,8 +418,10 @@ DLM_API int dlm_kernel_error(int* flag);
  *           automatic choice uses them on more than 128 nodes when x, m and their rows are aligned to
  *           32 bytes and d is a multiple of 8)
  * Results do not depend on the knobs, with one exception: the merged-staging kernels (knob 7 = 2 or 3,
- * the default on long rows: 8 or more entries; 12 or more for dsgd_step above 128 nodes) arrange the same
- * sum differently and agree with the other paths, and with each other, to rounding, not bitwise.
+ * the default from about 5 entries per row on, and for dmsgd_step / dsgd_step on most graphs of 12 nodes
+ * or more) arrange the same sum differently and agree with the other paths, and with each other, to
+ * rounding (relative L2 <= 1e-6), not bitwise.  Which kernel a call takes depends on n, the rows' lengths,
+ * the gradient type and the alignment, never on the values.
  * DLM_ERR_KIND for an unknown knob.
  */
 DLM_API int dlm_set_tuning(int knob, int value);
