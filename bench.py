@@ -194,7 +194,10 @@ def workload_config(args, w, n, d, world, g_esz):
                         (f" (tuning {args.tuning})" if args.tuning else ""),
             "n": n, "d": d, "topology": w.topology, "g_dtype": w.g_dtype, "beta": w.beta, "gamma": w.gamma,
             "parallelism": "replicas only" if world > 1 else "1 gpu",
-            "l2": f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"}
+            "l2": (f"working set {(8 + g_esz) * n * d / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"
+                   if (8 + g_esz) * n * d > 126e6 else
+                   f"working set {(8 + g_esz) * n * d / 1e6:.2f} MB per step fits the 126 MB L2 and is not flushed: "
+                   "an L2-resident, launch-bound timing, not an HBM figure")}
 
 
 def oracle_sample(workload, budget_s=20.0, steps=None, warmup=0, wall_limit_s=150.0):
